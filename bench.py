@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the SlideDP reduce + AdamW hot path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]            # libslidedp (CUDA)
+  python bench.py --impl reference [--steps K] [--warmup W]      # the CPU oracle, as it stands
+
+One "step" is one pass of the whole hot path over one Qwen3-8B-shaped decoder layer
+(192,946,176 parameters, R = 4 BF16 rank gradients, step 11, clip 1.0): the global-norm
+pass over all gradients, then the fused rank-reduce + AdamW + BF16-emit kernel.
+`value` is whole-job G-params/s with everything resident in HBM; `e2e` is the same step
+through slidedp_stream_step with the FP32 state in pinned HOST memory, host<->device copies
+inside the timed region. With --gpus N every rank updates its own layer (independent
+partitions, no data-path collective): weak scaling. Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "G-params/s per reduce+AdamW step"
+UNIT = "G-params/s"
+WORKLOAD = "qwen3_8b_layer"
+HOST_WORKLOAD = "qwen3_14b_layer_host"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per parameter of the fused update kernel, from
+# the ncu capture summarised in profiles/reduce_adamw_kernel_R4.md (None until captured).
+NCU_TRAFFIC_BYTES_PER_PARAM = None
+
+
+def measured_peak_hbm():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while running."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc, self.thread = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()          # this exact child, nothing else
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            if self.thread:
+                self.thread.join(timeout=2)
+        sm, smax, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); smax = float(r[1])
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": smax, "reasons": [], "samples": 0}
+        busy = [x for x in sm if x >= 0.5 * max(sm)]
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": smax,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- reference arm
+def run_reference(args):
+    """Times the CPU oracle, unchanged, on the host cores: each step is the whole path (norm +
+    update) over a bounded sample (the first 2^25 parameters) of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_2609_34162_b200 import workloads as W
+    wl = W.CONFIGS[WORKLOAD]
+    n = min(wl.numel, 1 << 25)
+    cores = min(len(os.sched_getaffinity(0)), oracle.max_threads())
+
+    def u16(t):
+        return t.view(torch.int16).numpy().view(np.uint16)
+    grads = [u16(W.rank_gradient(wl, r, step=wl.first_step)[:n].contiguous()) for r in range(wl.R)]
+    w = W.master_weights(wl)[:n].contiguous().numpy()
+    m, v, p = np.zeros(n, np.float32), np.zeros(n, np.float32), np.zeros(n, np.uint16)
+    t = 1
+    for _ in range(args.warmup):
+        oracle.step(grads, w, m, v, p, oracle.HParams(inv_R=1.0 / wl.R, max_norm=wl.max_norm,
+                                                      step=t, **wl.hparams), nthreads=cores)
+        t += 1
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.step(grads, w, m, v, p, oracle.HParams(inv_R=1.0 / wl.R, max_norm=wl.max_norm,
+                                                      step=t, **wl.hparams), nthreads=cores)
+        t += 1
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt / 1e9
+    sample = f"first {n} of {wl.numel} parameters per step, R={wl.R}, norm + update"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "params": wl.numel, "R": wl.R, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+    return 0
+
+
+# --------------------------------------------------------------------------------- CUDA arm
+def run_cuda(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_34162_b200.slidedp as sd          # raises if libslidedp.so is missing
+    from paper_2609_34162_b200 import workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libslidedp has no CPU path "
+                         "(use --impl reference for the CPU oracle)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    wl = W.CONFIGS[WORKLOAD]
+    n, R = wl.numel, wl.R
+    layer = rank                                   # every rank owns a different layer
+    ctx = sd.slidedp_create(local, 0)
+    stream = torch.cuda.current_stream()
+    dev = torch.device("cuda", local)
+
+    # ---- inputs, resident in HBM: R gradients of the measured step, FP32 state, BF16 out
+    t_meas = wl.first_step
+    grads = [W.rank_gradient(wl, r, step=t_meas, layer=layer, device=dev) for r in range(R)]
+    w = W.master_weights(wl, layer=layer, device=dev)
+    m = torch.zeros(n, device=dev)
+    v = torch.zeros(n, device=dev)
+    p = torch.zeros(n, dtype=torch.bfloat16, device=dev)
+
+    def hp(t):
+        return sd.HParams(inv_R=1.0 / R, max_norm=wl.max_norm, step=t, **wl.hparams)
+
+    def device_step(t, ev=None):
+        if ev: ev[0].record(stream)
+        ctx.slidedp_grad_norm(grads, n, 1.0 / R, True)
+        ctx.slidedp_grad_norm_finish(wl.max_norm)
+        if ev: ev[1].record(stream)
+        ctx.slidedp_reduce_adamw_chunk(grads, n, w, m, v, p, hp(t))
+        if ev: ev[2].record(stream)
+
+    # moments pre-warmed by the seeded steps that precede the measured one (timing only: the
+    # parity tests pre-warm with the oracle); fresh gradients each pre-warm step
+    tmp = [torch.empty(n, dtype=torch.bfloat16, device=dev) for _ in range(R)]
+    keep = grads
+    for t in range(1, wl.prewarm_steps + 1):
+        for r in range(R):
+            W.rank_gradient(wl, r, step=t, layer=layer, device=dev, out=tmp[r])
+        grads = tmp
+        device_step(t)
+    grads = keep
+    del tmp
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+
+    for i in range(max(args.warmup, 3)):
+        device_step(t_meas + i)
+    t_next = t_meas + max(args.warmup, 3)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = ctx.slidedp_kernel_launches()
+    barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record(stream)
+    for i in range(args.steps):
+        device_step(t_next + i, events[i])
+    stop.record(stream)
+    barrier()
+    launches = ctx.slidedp_kernel_launches() - launches0
+    total_ms = max_over_ranks(start.elapsed_time(stop))
+    norm_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in events)
+    upd_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in events)
+    upd_best = min(e[1].elapsed_time(e[2]) for e in events)
+    t_next += args.steps
+    clocks = sampler.stop() if rank == 0 else None
+
+    ms_per_step = total_ms / args.steps
+    value = world * n / (ms_per_step * 1e-3) / 1e9
+    peak, peak_kind = measured_peak_hbm()
+    upd_bytes = (26 + 2 * R) * n
+    achieved = upd_bytes / (upd_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "reduce_adamw_kernel<R=4>", "achieved": achieved,
+                "peak": peak, "peak_source": f"of {peak_kind}", "unit": "GB/s",
+                "frac": achieved / peak,
+                "traffic": (NCU_TRAFFIC_BYTES_PER_PARAM * n
+                            if NCU_TRAFFIC_BYTES_PER_PARAM is not None else None),
+                "algorithmic_bytes_per_launch": upd_bytes, "ms_per_launch": upd_ms,
+                "ms_per_launch_best": upd_best,
+                "frac_of_nominal_8000": achieved / 8000.0,
+                "norm_pass": {"ms": norm_ms, "algorithmic_bytes": 2 * R * n,
+                              "achieved": 2 * R * n / (norm_ms * 1e-3) / 1e9,
+                              "frac": 2 * R * n / (norm_ms * 1e-3) / 1e9 / peak}}
+
+    # ---- e2e: the same step with the FP32 state in pinned host memory ------------------
+    ce = W.chunk_elems(64)
+    hw = torch.empty(n, pin_memory=True); hm = torch.empty(n, pin_memory=True)
+    hv = torch.empty(n, pin_memory=True)
+    hw.copy_(w); hm.copy_(m); hv.copy_(v)
+    torch.cuda.synchronize()
+    for i in range(2):
+        ctx.slidedp_stream_step(grads, n, hw, hm, hv, p, ce, 3, hp(t_next + i), want_stats=False)
+    t_next += 2
+    e2e_steps = max(1, min(args.steps, 10))
+    barrier()
+    e2e_ms, wall0, last = 0.0, time.perf_counter(), None
+    for i in range(e2e_steps):
+        last = ctx.slidedp_stream_step(grads, n, hw, hm, hv, p, ce, 3, hp(t_next + i))
+        e2e_ms += last["ms_total"]
+    wall = time.perf_counter() - wall0
+    barrier()
+    t_next += e2e_steps
+    e2e_ms = max_over_ranks(e2e_ms)
+    e2e = {"value": world * n * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+           "h2d_bytes_per_step": 12 * n, "d2h_bytes_per_step": 12 * n + 32,
+           "ms_per_step": e2e_ms / e2e_steps, "wall_ms_per_step": wall / e2e_steps * 1e3,
+           "steps": e2e_steps, "chunk_mib": 64, "nbuf": 3,
+           "note": "FP32 master/m/v in pinned host memory, copied H2D and back D2H every step; "
+                   "gradients and the BF16 copy stay on the device where backward/forward use them",
+           "link_gbs_h2d": last["gbs_h2d"], "link_gbs_d2h": last["gbs_d2h"]}
+    del hw, hm, hv
+
+    out = None
+    if rank == 0:
+        # ---- host-resident configuration proper + the measured host-link roofline ------
+        host = None
+        try:
+            host = host_resident_report(ctx, sd, W, torch, dev)
+        except Exception as exc:                       # report, never hide
+            host = {"error": repr(exc)}
+        cpu = cpu_baseline(W, torch, np, wl, grads, layer)
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "params_per_gpu": n, "R": R, "step": t_meas,
+                       "clip_max_norm": wl.max_norm, "mode": "device-resident",
+                       "parallelism": f"{world} independent layer(s), one per GPU, no collective",
+                       "l2": "inputs (8.1 GB touched per step) exceed the 126 MB L2"},
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+            "clocks": clocks, "host_resident": host,
+        }
+    ctx.slidedp_destroy()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if out is not None:
+        print(json.dumps(out))
+    return 0
+
+
+def host_resident_report(ctx, sd, W, torch, dev):
+    """Qwen3-14B-shaped layer with pinned host state, 64 MiB chunks, 3 slots, against the
+    pinned-copy bandwidth measured in the same run."""
+    wl = W.CONFIGS[HOST_WORKLOAD]
+    n, R = wl.numel, wl.R
+    grads = [W.rank_gradient(wl, r, step=wl.first_step, device=dev) for r in range(R)]
+    p = torch.zeros(n, dtype=torch.bfloat16, device=dev)
+    hw = torch.empty(n, pin_memory=True); hm = torch.empty(n, pin_memory=True)
+    hv = torch.empty(n, pin_memory=True)
+    hw.copy_(W.master_weights(wl, device=dev)); hm.zero_(); hv.zero_()
+    # link probe on 1 GiB per direction in 64 MiB copies, reusing hw/hm as the pinned buffers
+    dbuf = torch.empty(2 << 28, dtype=torch.float32, device=dev)
+    probe = ctx.slidedp_link_probe(hw, hm, dbuf[:1 << 28], dbuf[1 << 28:], 1 << 30, 64 << 20, 3)
+    del dbuf
+    hw.copy_(W.master_weights(wl, device=dev)); hm.zero_()
+    torch.cuda.synchronize()
+    ce = W.chunk_elems(64)
+    runs = []
+    for i in range(5):
+        st = ctx.slidedp_stream_step(grads, n, hw, hm, hv, p, ce, 3,
+                                     sd.HParams(inv_R=1.0 / R, max_norm=wl.max_norm, step=1 + i,
+                                                **wl.hparams))
+        if i >= 2:
+            runs.append(st)
+    ms = statistics.mean(r["ms_total"] for r in runs)
+    link_bytes = 12.0 * n
+    bound_ms = max(link_bytes / (probe["h2d_bidir"] * 1e6), link_bytes / (probe["d2h_bidir"] * 1e6))
+    return {"workload": HOST_WORKLOAD, "params": n, "R": R, "chunk_mib": 64, "nbuf": 3,
+            "value": n / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
+            "link_probe_gbs": probe,
+            "link_gbs_effective_each_way": link_bytes / (ms * 1e6),
+            "roofline": {"bound": "host-link", "unit": "GB/s",
+                         "achieved": link_bytes / (ms * 1e6),
+                         "peak": min(probe["h2d_bidir"], probe["d2h_bidir"]),
+                         "frac": bound_ms / ms,
+                         "peak_source": "pinned-copy probe in this run, both directions at once"},
+            "lanes_ms": {k: statistics.mean(r[k] for r in runs)
+                         for k in ("ms_norm", "ms_h2d", "ms_kernel", "ms_d2h")}}
+
+
+def cpu_baseline(W, torch, np, wl, grads, layer):
+    """The oracle as it stands, one whole step (norm + update) of the same layer on the host
+    cores of this machine."""
+    import oracle
+    cores = min(len(os.sched_getaffinity(0)), oracle.max_threads())
+    n = wl.numel if cores >= 4 else wl.numel // 4
+    hg = [g[:n].cpu().view(torch.int16).numpy().view(np.uint16) for g in grads]
+    w = W.master_weights(wl, layer=layer)[:n].contiguous().numpy()
+    m, v, p = np.zeros(n, np.float32), np.zeros(n, np.float32), np.zeros(n, np.uint16)
+    kw = dict(inv_R=1.0 / wl.R, max_norm=wl.max_norm, **wl.hparams)
+    oracle.step([g[:1 << 20] for g in hg], w[:1 << 20], m[:1 << 20], v[:1 << 20], p[:1 << 20],
+                oracle.HParams(step=1, **kw), nthreads=cores)           # warm the threads
+    t0 = time.perf_counter()
+    oracle.step(hg, w, m, v, p, oracle.HParams(step=2, **kw), nthreads=cores)
+    dt = time.perf_counter() - t0
+    return {"value": n / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"one whole step (norm + update) over {n} of {wl.numel} parameters, R={wl.R}",
+            "seconds": dt}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_cuda(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,179 @@
+/*
+ * slidedp.h -- C ABI of libslidedp: the data-parallel hot path of SlideDP's synchronous
+ * step on one B200 (sm_100a).
+ *
+ * For each flat parameter chunk the library sums R rank-gradient BF16 buffers in a fixed
+ * rank order with FP32 accumulation, scales by 1/R, optionally applies a deterministic
+ * global-L2-norm clip, runs AdamW over the single authoritative FP32 master / m / v state
+ * and emits the BF16 parameter copy for the next delivery. The paper runs this step on
+ * host CPUs (Sec. 3.2 "Gradient return", Sec. 3.3 Reduce -> D2H -> Adam); here it is one
+ * fused streaming kernel per chunk, with the state either resident in HBM or resident in
+ * pinned host memory and streamed through a small ring of device slots.
+ *
+ * State per parameter (paper Sec. 2.1, Table 1): BF16 parameter 2 B, BF16 gradient 2 B,
+ * FP32 master 4 B, FP32 m 4 B, FP32 v 4 B = 16 B.
+ *
+ * Conventions
+ *  - Every function returns SLIDEDP_OK (0) or a negative slidedp_status; nothing throws,
+ *    aborts or exits. slidedp_strerror() names a status; slidedp_last_cuda_error() gives
+ *    the cudaError_t behind SLIDEDP_ERR_CUDA.
+ *  - The caller owns every data buffer and passes raw pointers; "device" pointers are
+ *    cudaMalloc'd (or torch) addresses on the context's device, "host" pointers are plain
+ *    host addresses, "pinned" pointers are page-locked host addresses. The library
+ *    allocates only inside slidedp_ctx (norm partials, scalars, streaming slots, streams,
+ *    events) and keeps nothing else between calls.
+ *  - BF16 buffers are arrays of 16-bit patterns. Every gradient / state / output base
+ *    pointer must be 16-byte aligned (SLIDEDP_ERR_MISALIGNED otherwise); n may be any
+ *    non-negative count (a ragged tail is handled element by element; n = 0 is a no-op).
+ *  - cuda_stream arguments are cudaStream_t handles passed as void* (NULL = legacy
+ *    default stream). Device-resident calls only enqueue work on that stream and return.
+ *  - master / m / v are updated in place; gradients are read-only; param_bf16_out must
+ *    not overlap any other argument.
+ */
+#ifndef SLIDEDP_H
+#define SLIDEDP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SLIDEDP_MAX_RANKS 16
+
+#if defined(__GNUC__)
+#define SLIDEDP_API __attribute__((visibility("default")))
+#else
+#define SLIDEDP_API
+#endif
+
+typedef enum {
+  SLIDEDP_OK = 0,
+  SLIDEDP_ERR_INVALID_ARG = -1, /* null pointer, R outside 1..16, n < 0, step < 1, beta outside [0,1), ... */
+  SLIDEDP_ERR_MISALIGNED = -2,  /* a base pointer is not 16-byte aligned                               */
+  SLIDEDP_ERR_BUDGET = -3,      /* the streaming slots would not fit the context's GPU memory budget   */
+  SLIDEDP_ERR_NOT_PINNED = -4,  /* a host state pointer of slidedp_stream_step is not page-locked      */
+  SLIDEDP_ERR_CUDA = -5,        /* a CUDA runtime call failed; see slidedp_last_cuda_error()            */
+  SLIDEDP_ERR_TIMEOUT = -6,     /* a bounded wait for queued work expired                               */
+  SLIDEDP_ERR_NO_NORM = -7      /* clipping requested but no finished norm is held by the context      */
+} slidedp_status;
+
+typedef struct slidedp_ctx slidedp_ctx;
+
+/* Hyper-parameters of one update. All doubles: float-typed constants alone (0.9f, 1-0.9f)
+ * already break a 1e-6 relative tolerance on m. */
+typedef struct {
+  double lr, beta1, beta2, eps, weight_decay;
+  double inv_R;    /* the FP32 rank sum is multiplied by (float)inv_R                        */
+  double max_norm; /* > 0: scale the averaged gradient by the context's clip coefficient      */
+  int64_t step;    /* 1-based index of the update being performed (bias correction uses it)  */
+} slidedp_hparams;
+
+/* What slidedp_stream_step measured (CUDA events; times in ms, rates in GB/s = 1e9 B/s). */
+typedef struct {
+  double norm, clip_coef; /* the step's global norm and coefficient (0 and 1 if clipping off) */
+  double ms_total;        /* first enqueue to last D2H complete                                */
+  double ms_norm;         /* the norm pass when it ran inside the call                         */
+  double ms_h2d, ms_kernel, ms_d2h; /* summed busy time of each lane over all chunks          */
+  double gbs_h2d, gbs_d2h;          /* bytes moved / summed busy time of that lane            */
+  int64_t chunks;
+  int32_t nonfinite;      /* 1 if the norm was inf or NaN                                      */
+  int32_t reserved;
+} slidedp_stats;
+
+/* ---- context ------------------------------------------------------------------------ */
+
+/* Creates a context on `device`. gpu_budget_bytes caps what slidedp_stream_step may allocate
+ * for its slots (0 = no cap). Allocates the norm workspace (a few MB) and three streams. */
+SLIDEDP_API int slidedp_create(slidedp_ctx** out, int device, size_t gpu_budget_bytes);
+/* Waits (bounded) for the context's own streams, frees everything. NULL is a no-op. */
+SLIDEDP_API int slidedp_destroy(slidedp_ctx* ctx);
+SLIDEDP_API const char* slidedp_strerror(int status);
+SLIDEDP_API int slidedp_last_cuda_error(const slidedp_ctx* ctx);
+
+/* Paper Sec. 2.1 / Table 1: bytes of persistent state for n parameters = 16 n. */
+SLIDEDP_API size_t slidedp_state_bytes(int64_t n);
+
+/* ---- global L2 norm of the averaged gradient (clipping; not part of the paper) --------
+ *
+ * slidedp_grad_norm adds, for one chunk, the sum over i of gbar_i^2 to the context's
+ * accumulator, where gbar_i = fl32(fl32-sum over ranks in order 0..R-1 of g_r[i]) * (float)inv_R
+ * as in Sec. 3.2 "Gradient return" (sum, then average). Squares and sums are FP64. The chunk
+ * is cut into fixed tiles of 16384 elements; each tile is summed by a fixed tree into its
+ * own slot, so the result does not depend on the launch shape, and a step cut into chunks
+ * at multiples of 16384 elements gives bit-identical results to the uncut step.
+ * first_chunk != 0 restarts the accumulation. Call the chunks of a step in a fixed order on
+ * ONE stream (or order the streams yourself).
+ *
+ * slidedp_grad_norm_finish folds the tile sums in a fixed order and leaves, in device
+ * memory owned by the context, sumsq, norm = sqrt(sumsq) and
+ * coef = max_norm > 0 ? min(1, max_norm / (norm + 1e-6)) : 1. If host_norm / host_coef is
+ * non-NULL the call also waits (bounded) for the stream and returns the values.
+ */
+SLIDEDP_API int slidedp_grad_norm(slidedp_ctx* ctx, const void* const* grads_bf16 /* host array of R device ptrs */,
+                      int R, int64_t n, double inv_R, int first_chunk, void* cuda_stream);
+SLIDEDP_API int slidedp_grad_norm_finish(slidedp_ctx* ctx, double max_norm, double* host_norm /* nullable */,
+                             double* host_coef /* nullable */, void* cuda_stream);
+
+/* ---- device-resident update: one fused kernel per chunk -------------------------------
+ *
+ * For i in [0, n):   (Sec. 3.2: one update of the authoritative FP32 state per iteration
+ *                     from the rank-averaged gradient; Sec. 3.3: the BF16 copy is a cast
+ *                     of the FP32 master)
+ *   gbar = fl32( ((g_0[i] + g_1[i]) + ... + g_{R-1}[i]) in FP32 ) * (float)inv_R
+ *   g    = gbar * c          c = context's clip coefficient if hp->max_norm > 0, else 1
+ *   m'   = beta1 m + (1-beta1) g          v' = beta2 v + (1-beta2) g^2
+ *   w'   = w - lr * ( (m'/(1-beta1^t)) / (sqrt(v'/(1-beta2^t)) + eps) + weight_decay * w )
+ *   master[i], m[i], v[i] = fl32(w'), fl32(m'), fl32(v')      (FP64 arithmetic, one rounding)
+ *   param_bf16_out[i] = bf16_round_to_nearest_even(master[i])
+ * grads_bf16: host array of R device pointers to n BF16 values each. master, m, v: device,
+ * n floats, in place. param_bf16_out: device, n BF16 values. When hp->max_norm > 0 a
+ * slidedp_grad_norm_finish must have been enqueued earlier on the same stream
+ * (SLIDEDP_ERR_NO_NORM if none was ever issued on this context).
+ * Asynchronous on cuda_stream; traffic is 26 + 2R bytes per parameter.
+ */
+SLIDEDP_API int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                               float* master, float* m, float* v, void* param_bf16_out,
+                               const slidedp_hparams* hp, void* cuda_stream);
+
+/* ---- host-resident update: state in pinned host memory, streamed chunk by chunk -------
+ *
+ * host_master / host_m / host_v: PINNED host arrays of n_total floats, updated in place.
+ * grads_bf16 (R device pointers, n_total each) and param_bf16_out (device, n_total) stay on
+ * the device. The step is cut every chunk_elems parameters (a multiple of 8; the last chunk
+ * may be short). Chunk k uses slot k mod nbuf (nbuf = 2 or 3): its three state arrays are
+ * copied H2D on a copy-in stream, updated by the fused kernel on a compute stream and copied
+ * back D2H on a copy-out stream, so that copy-in, kernel and copy-out of different chunks
+ * overlap (Sec. 3.3 "Overlap within a layer"); a slot is reused only after its copy-out has
+ * completed (Sec. 3.3 "Completion and buffer reuse"). Slots take nbuf * 3 * chunk_elems * 4
+ * bytes of device memory inside the context and must fit its budget (SLIDEDP_ERR_BUDGET,
+ * before any work). If hp->max_norm > 0 and norm_ready == 0 the call first computes the
+ * global norm over these n_total gradients; with norm_ready != 0 it uses the coefficient
+ * already held by the context (a step that spans several calls: run slidedp_grad_norm over
+ * every layer and slidedp_grad_norm_finish first). Synchronous: returns after the last
+ * copy-out completed (bounded wait, SLIDEDP_ERR_TIMEOUT). stats is nullable.
+ * Link traffic is 12 bytes per parameter in each direction.
+ */
+SLIDEDP_API int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n_total,
+                        float* host_master, float* host_m, float* host_v,
+                        void* param_bf16_out, int64_t chunk_elems, int nbuf, int norm_ready,
+                        const slidedp_hparams* hp, slidedp_stats* stats);
+
+/* ---- host-link probe: the roofline of the host-resident mode ---------------------------
+ *
+ * Copies `bytes` between a pinned host buffer and a device buffer in pieces of copy_bytes,
+ * reps times, and reports GB/s: out4[0] H2D alone, out4[1] D2H alone, out4[2] / out4[3] H2D
+ * and D2H while both run at once on two streams. host_a/host_b pinned, dev_a/dev_b device,
+ * each at least `bytes` long. Synchronous (bounded waits).
+ */
+SLIDEDP_API int slidedp_link_probe(slidedp_ctx* ctx, void* host_a, void* host_b, void* dev_a, void* dev_b,
+                       size_t bytes, size_t copy_bytes, int reps, double out4[4]);
+
+/* Number of kernels this library has launched on the context since creation. */
+SLIDEDP_API int64_t slidedp_kernel_launches(const slidedp_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,285 @@
+// Device kernels of libslidedp (sm_100a): the fused rank-reduce + AdamW + BF16-emit
+// streaming kernel, and the two-pass fixed-tree sum of squares behind the global norm.
+//
+// The path is elementwise and HBM-bound (26 + 2R bytes per parameter), so there are no
+// tensor cores here: each thread owns 8 consecutive parameters, moves them with 128-bit
+// accesses, keeps everything in registers and stores each output once.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace slidedp {
+
+constexpr int kMaxRanks = 16;
+constexpr int kVec = 8;                 // parameters per thread per group (one 16-byte BF16 load)
+constexpr int kUpdateThreads = 256;
+constexpr int kNormThreads = 256;
+constexpr int kNormIters = 8;
+constexpr int kNormTile = kNormThreads * kVec * kNormIters;   // 16384 elements per partial
+constexpr int kFinishThreads = 1024;
+
+struct GradPtrs {
+  const uint16_t* p[kMaxRanks];
+};
+
+// Everything the update needs that does not depend on the element, prepared on the host
+// in double from the double-typed hyper-parameters.
+struct UpdateConsts {
+  double beta1, beta2;
+  double omb1, omb2;        // 1 - beta1, 1 - beta2 (exact in double for beta in [0.5, 1))
+  double rsqrt_bc2;         // 1 / sqrt(1 - beta2^t)
+  double eps;
+  double neg_lr_over_bc1;   // -lr / (1 - beta1^t)
+  double decay;             // 1 - lr * weight_decay
+  float inv_R;              // (float)inv_R
+};
+
+// ---- small helpers -----------------------------------------------------------------
+
+__device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xFFFF0000u); }
+
+// FP32 -> BF16 bits, round to nearest even, NaN stays NaN.
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float x) {
+  uint16_t r;
+  asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(x));
+  return (uint32_t)r;
+}
+
+// Streaming (read-once / write-once) 128-bit accesses: keep them out of L1 and mark them
+// evict-first in L2, since nothing on this path is ever re-read.
+__device__ __forceinline__ uint4 ld_stream(const void* p) {
+  return __ldcs(reinterpret_cast<const uint4*>(p));
+}
+__device__ __forceinline__ void st_stream(void* p, uint4 v) {
+  __stcs(reinterpret_cast<uint4*>(p), v);
+}
+
+// Hardware seeds for FP64 reciprocal square root and reciprocal (about 20 good bits; the
+// full double exponent range). One Newton step each below brings them to ~1e-12.
+__device__ __forceinline__ double rsqrt_seed(double x) {
+  double r;
+  asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(r) : "d"(x));
+  return r;
+}
+__device__ __forceinline__ double rcp_seed(double x) {
+  double r;
+  asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(r) : "d"(x));
+  return r;
+}
+
+// Averaged gradient of one element: left-to-right FP32 sum over the ranks, times (float)1/R.
+// `vals` holds the R rank values in rank order.
+template <int R>
+__device__ __forceinline__ float rank_mean(const float (&vals)[R], float inv_R) {
+  float s = vals[0];
+#pragma unroll
+  for (int r = 1; r < R; ++r) s = __fadd_rn(s, vals[r]);
+  return __fmul_rn(s, inv_R);
+}
+
+// One parameter's AdamW update in FP64 from the FP32 state. k1 = (1-beta1) c and
+// k2 = (1-beta2) c^2 carry the clip coefficient c.
+__device__ __forceinline__ void adamw_element(float gbar, float& w, float& m, float& v,
+                                              const UpdateConsts& k, double k1, double k2) {
+  const double g = (double)gbar;
+  const double m1 = fma(k.beta1, (double)m, k1 * g);
+  const double v1 = fma(k.beta2, (double)v, k2 * (g * g));     // g*g is exact in double
+  // s = sqrt(v1): seed, then one Newton step on the root itself.
+  const double r = v1 > 0.0 ? rsqrt_seed(v1) : 0.0;
+  double s = v1 * r;
+  s = fma(fma(-s, s, v1), 0.5 * r, s);
+  if (!(v1 < 1.7976931348623157e308)) s = v1;                  // +inf and NaN pass through
+  const double d = fma(s, k.rsqrt_bc2, k.eps);                 // sqrt(v1/bc2) + eps
+  // q = m1 / d: seed reciprocal, one correction of the quotient.
+  const double rc = rcp_seed(d);
+  double q = m1 * rc;
+  q = fma(fma(-q, d, m1), rc, q);
+  if (!(d > 0.0) || !(d < 1.7976931348623157e308)) q = m1 / d; // 0, inf, NaN: IEEE division
+  const double w1 = fma(k.neg_lr_over_bc1, q, k.decay * (double)w);
+  m = __double2float_rn(m1);
+  v = __double2float_rn(v1);
+  w = __double2float_rn(w1);
+}
+
+// ---- fused update kernel -------------------------------------------------------------
+//
+// R_T > 0: rank count known at compile time (loads fully unrolled). R_T == 0: runtime R.
+template <int R_T>
+__global__ void __launch_bounds__(kUpdateThreads)
+reduce_adamw_kernel(GradPtrs gp, int R_rt, int64_t n, float* __restrict__ master,
+                    float* __restrict__ mom1, float* __restrict__ mom2,
+                    uint16_t* __restrict__ param_out, UpdateConsts k,
+                    const double* __restrict__ clip_coef) {
+  const int R = R_T > 0 ? R_T : R_rt;
+  const int64_t base = ((int64_t)blockIdx.x * kUpdateThreads + threadIdx.x) * kVec;
+  if (base >= n) return;
+  const double c = clip_coef ? *clip_coef : 1.0;
+  const double k1 = k.omb1 * c, k2 = k.omb2 * c * c;
+
+  if (base + kVec <= n) {
+    // issue every load of this thread before the first use
+    uint4 graw[R_T > 0 ? R_T : kMaxRanks];
+#pragma unroll
+    for (int r = 0; r < (R_T > 0 ? R_T : kMaxRanks); ++r)
+      if (r < R) graw[r] = ld_stream(gp.p[r] + base);
+    uint4 wq[2], mq[2], vq[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      wq[h] = ld_stream(master + base + 4 * h);
+      mq[h] = ld_stream(mom1 + base + 4 * h);
+      vq[h] = ld_stream(mom2 + base + 4 * h);
+    }
+    float s[kVec];
+    {
+      const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[0]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { s[2 * j] = bf16_lo(x[j]); s[2 * j + 1] = bf16_hi(x[j]); }
+    }
+#pragma unroll
+    for (int r = 1; r < (R_T > 0 ? R_T : kMaxRanks); ++r) {
+      if (r < R) {
+        const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[r]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          s[2 * j] = __fadd_rn(s[2 * j], bf16_lo(x[j]));
+          s[2 * j + 1] = __fadd_rn(s[2 * j + 1], bf16_hi(x[j]));
+        }
+      }
+    }
+    float* wf = reinterpret_cast<float*>(wq);
+    float* mf = reinterpret_cast<float*>(mq);
+    float* vf = reinterpret_cast<float*>(vq);
+    uint32_t pb[kVec];
+#pragma unroll
+    for (int j = 0; j < kVec; ++j) {
+      adamw_element(__fmul_rn(s[j], k.inv_R), wf[j], mf[j], vf[j], k, k1, k2);
+      pb[j] = f32_to_bf16_bits(wf[j]);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      st_stream(master + base + 4 * h, wq[h]);
+      st_stream(mom1 + base + 4 * h, mq[h]);
+      st_stream(mom2 + base + 4 * h, vq[h]);
+    }
+    uint4 pq;
+    pq.x = pb[0] | (pb[1] << 16); pq.y = pb[2] | (pb[3] << 16);
+    pq.z = pb[4] | (pb[5] << 16); pq.w = pb[6] | (pb[7] << 16);
+    st_stream(param_out + base, pq);
+  } else {
+    // ragged tail: fewer than 8 parameters left, one at a time
+    for (int64_t i = base; i < n; ++i) {
+      float s = __uint_as_float((uint32_t)gp.p[0][i] << 16);
+      for (int r = 1; r < R; ++r) s = __fadd_rn(s, __uint_as_float((uint32_t)gp.p[r][i] << 16));
+      float w = master[i], m = mom1[i], v = mom2[i];
+      adamw_element(__fmul_rn(s, k.inv_R), w, m, v, k, k1, k2);
+      master[i] = w; mom1[i] = m; mom2[i] = v;
+      param_out[i] = (uint16_t)f32_to_bf16_bits(w);
+    }
+  }
+}
+
+// ---- sum of squares of the averaged gradient ----------------------------------------------
+//
+// Pass 1: one FP64 partial per fixed tile of kNormTile elements. Inside a tile thread t
+// adds its 8 * kNormIters squares in index order, the warp folds by an xor butterfly
+// (16, 8, 4, 2, 1), and thread 0 adds the 8 warp sums in warp order: the tree is fixed, so
+// a tile's partial does not depend on which block computes it or on the grid size.
+template <int R_T>
+__global__ void __launch_bounds__(kNormThreads)
+grad_sumsq_tiles_kernel(GradPtrs gp, int R_rt, int64_t n, float inv_R,
+                        double* __restrict__ partials) {
+  const int R = R_T > 0 ? R_T : R_rt;
+  __shared__ double warp_sum[kNormThreads / 32];
+  const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
+  for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    const int64_t tbase = tile * kNormTile + (int64_t)threadIdx.x * kVec;
+    double acc = 0.0;
+#pragma unroll 4
+    for (int it = 0; it < kNormIters; ++it) {
+      const int64_t e = tbase + (int64_t)it * (kNormThreads * kVec);
+      float s[kVec];
+      if (e + kVec <= n) {
+        uint4 graw[R_T > 0 ? R_T : kMaxRanks];
+#pragma unroll
+        for (int r = 0; r < (R_T > 0 ? R_T : kMaxRanks); ++r)
+          if (r < R) graw[r] = ld_stream(gp.p[r] + e);
+        {
+          const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[0]);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) { s[2 * j] = bf16_lo(x[j]); s[2 * j + 1] = bf16_hi(x[j]); }
+        }
+#pragma unroll
+        for (int r = 1; r < (R_T > 0 ? R_T : kMaxRanks); ++r) {
+          if (r < R) {
+            const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[r]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              s[2 * j] = __fadd_rn(s[2 * j], bf16_lo(x[j]));
+              s[2 * j + 1] = __fadd_rn(s[2 * j + 1], bf16_hi(x[j]));
+            }
+          }
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < kVec; ++j) {
+          s[j] = 0.0f;
+          if (e + j < n) {
+            float t = __uint_as_float((uint32_t)gp.p[0][e + j] << 16);
+            for (int r = 1; r < R; ++r)
+              t = __fadd_rn(t, __uint_as_float((uint32_t)gp.p[r][e + j] << 16));
+            s[j] = t;
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < kVec; ++j) {
+        const double g = (double)__fmul_rn(s[j], inv_R);
+        acc = fma(g, g, acc);
+      }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+    if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double t = warp_sum[0];
+#pragma unroll
+      for (int w = 1; w < kNormThreads / 32; ++w) t += warp_sum[w];
+      partials[tile] = t;
+    }
+    __syncthreads();
+  }
+}
+
+// Pass 2: one block folds `count` partials in a fixed order: thread t adds partials
+// t, t + 1024, ... in that order, then the same warp butterfly and warp-order sum.
+// Writes scalars[0] = sumsq, [1] = norm, [2] = clip coefficient, [3] = 1.0 if non-finite.
+__global__ void __launch_bounds__(kFinishThreads)
+grad_norm_finish_kernel(const double* __restrict__ partials, int64_t count, double max_norm,
+                        double* __restrict__ scalars) {
+  __shared__ double warp_sum[kFinishThreads / 32];
+  double acc = 0.0;
+  for (int64_t i = threadIdx.x; i < count; i += kFinishThreads) acc += partials[i];
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+  if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = warp_sum[0];
+    for (int w = 1; w < kFinishThreads / 32; ++w) t += warp_sum[w];
+    const double norm = sqrt(t);
+    double c = 1.0;
+    if (max_norm > 0.0) {
+      c = max_norm / (norm + 1e-6);
+      if (c > 1.0) c = 1.0;      // a NaN coefficient stays NaN
+    }
+    scalars[0] = t;
+    scalars[1] = norm;
+    scalars[2] = c;
+    scalars[3] = (norm - norm == 0.0) ? 0.0 : 1.0;
+  }
+}
+
+}  // namespace slidedp

@@ -1,0 +1,604 @@
+// libslidedp: C ABI over the sm_100a kernels in kernels.cuh. See include/slidedp.h for
+// the contract of every entry point. Host code here only validates arguments, prepares the
+// per-step constants in double, launches kernels and drives the host-resident slot ring.
+#include "slidedp.h"
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <string.h>
+#include <time.h>
+
+#include <new>
+#include <vector>
+
+#include "kernels.cuh"
+
+using namespace slidedp;
+
+namespace {
+
+constexpr double kWaitSeconds = 300.0;       // bound on every host-side wait
+constexpr int64_t kInitialPartials = 1 << 20;  // 8 MB: 2^20 tiles = 17 G parameters
+
+struct ChunkEvents {
+  cudaEvent_t h2d_start, h2d_end, k_start, k_end, d2h_start, d2h_end;
+};
+
+}  // namespace
+
+struct slidedp_ctx {
+  int device = 0;
+  size_t budget = 0;
+  int last_cuda = 0;
+  int64_t launches = 0;
+  // norm workspace
+  double* partials = nullptr;
+  int64_t partials_cap = 0;
+  int64_t partials_used = 0;
+  double* scalars = nullptr;        // device: sumsq, norm, coef, nonfinite
+  double* host_scalars = nullptr;   // pinned mirror
+  bool norm_issued = false;
+  cudaEvent_t scalar_event = nullptr;
+  // host-resident streaming
+  cudaStream_t s_in = nullptr, s_compute = nullptr, s_out = nullptr;
+  float* slots = nullptr;
+  size_t slot_bytes = 0;            // bytes currently allocated for all slots
+  cudaEvent_t ev_loaded[3] = {nullptr, nullptr, nullptr};
+  cudaEvent_t ev_updated[3] = {nullptr, nullptr, nullptr};
+  cudaEvent_t ev_free[3] = {nullptr, nullptr, nullptr};
+  cudaEvent_t ev_begin = nullptr, ev_norm_done = nullptr, ev_end = nullptr;
+  std::vector<ChunkEvents> timing;  // grown on demand, reused
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+int cuda_fail(slidedp_ctx* ctx, cudaError_t e) {
+  if (ctx) ctx->last_cuda = (int)e;
+  (void)cudaGetLastError();
+  return SLIDEDP_ERR_CUDA;
+}
+
+#define CU(call)                                            \
+  do {                                                      \
+    cudaError_t e_ = (call);                                \
+    if (e_ != cudaSuccess) return cuda_fail(ctx, e_);       \
+  } while (0)
+
+double now_seconds() {
+  timespec ts;
+  clock_gettime(CLOCK_MONOTONIC, &ts);
+  return (double)ts.tv_sec + 1e-9 * (double)ts.tv_nsec;
+}
+
+// Waits for an event without ever blocking unboundedly inside the driver.
+int bounded_event_wait(slidedp_ctx* ctx, cudaEvent_t ev, double seconds) {
+  const double deadline = now_seconds() + seconds;
+  for (;;) {
+    cudaError_t e = cudaEventQuery(ev);
+    if (e == cudaSuccess) return SLIDEDP_OK;
+    if (e != cudaErrorNotReady) return cuda_fail(ctx, e);
+    if (now_seconds() > deadline) return SLIDEDP_ERR_TIMEOUT;
+    timespec nap = {0, 20000};
+    nanosleep(&nap, nullptr);
+  }
+}
+
+int bounded_stream_wait(slidedp_ctx* ctx, cudaStream_t s, double seconds) {
+  const double deadline = now_seconds() + seconds;
+  for (;;) {
+    cudaError_t e = cudaStreamQuery(s);
+    if (e == cudaSuccess) return SLIDEDP_OK;
+    if (e != cudaErrorNotReady) return cuda_fail(ctx, e);
+    if (now_seconds() > deadline) return SLIDEDP_ERR_TIMEOUT;
+    timespec nap = {0, 20000};
+    nanosleep(&nap, nullptr);
+  }
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_grads(const void* const* grads, int R, GradPtrs* out) {
+  if (!grads || R < 1 || R > SLIDEDP_MAX_RANKS) return SLIDEDP_ERR_INVALID_ARG;
+  for (int r = 0; r < kMaxRanks; ++r) out->p[r] = nullptr;
+  for (int r = 0; r < R; ++r) {
+    if (!grads[r]) return SLIDEDP_ERR_INVALID_ARG;
+    if (!aligned16(grads[r])) return SLIDEDP_ERR_MISALIGNED;
+    out->p[r] = static_cast<const uint16_t*>(grads[r]);
+  }
+  return SLIDEDP_OK;
+}
+
+int check_hparams(const slidedp_hparams* hp) {
+  if (!hp) return SLIDEDP_ERR_INVALID_ARG;
+  if (hp->step < 1) return SLIDEDP_ERR_INVALID_ARG;
+  if (!(hp->beta1 >= 0.0 && hp->beta1 < 1.0)) return SLIDEDP_ERR_INVALID_ARG;
+  if (!(hp->beta2 >= 0.0 && hp->beta2 < 1.0)) return SLIDEDP_ERR_INVALID_ARG;
+  if (!(hp->eps >= 0.0) || hp->lr != hp->lr || hp->weight_decay != hp->weight_decay ||
+      hp->inv_R != hp->inv_R)
+    return SLIDEDP_ERR_INVALID_ARG;
+  return SLIDEDP_OK;
+}
+
+UpdateConsts make_consts(const slidedp_hparams* hp) {
+  UpdateConsts k;
+  const double bc1 = 1.0 - pow(hp->beta1, (double)hp->step);
+  const double bc2 = 1.0 - pow(hp->beta2, (double)hp->step);
+  k.beta1 = hp->beta1;
+  k.beta2 = hp->beta2;
+  k.omb1 = 1.0 - hp->beta1;
+  k.omb2 = 1.0 - hp->beta2;
+  k.rsqrt_bc2 = 1.0 / sqrt(bc2);
+  k.eps = hp->eps;
+  k.neg_lr_over_bc1 = -hp->lr / bc1;
+  k.decay = 1.0 - hp->lr * hp->weight_decay;
+  k.inv_R = (float)hp->inv_R;
+  return k;
+}
+
+template <int R_T>
+void launch_update_t(const GradPtrs& gp, int R, int64_t n, float* w, float* m, float* v,
+                     uint16_t* p, const UpdateConsts& k, const double* coef, cudaStream_t st) {
+  const int64_t groups = (n + kVec - 1) / kVec;
+  const unsigned blocks = (unsigned)((groups + kUpdateThreads - 1) / kUpdateThreads);
+  reduce_adamw_kernel<R_T><<<blocks, kUpdateThreads, 0, st>>>(gp, R, n, w, m, v, p, k, coef);
+}
+
+int launch_update(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, float* w, float* m,
+                  float* v, uint16_t* p, const UpdateConsts& k, const double* coef,
+                  cudaStream_t st) {
+  if (n == 0) return SLIDEDP_OK;
+  switch (R) {
+    case 1: launch_update_t<1>(gp, R, n, w, m, v, p, k, coef, st); break;
+    case 2: launch_update_t<2>(gp, R, n, w, m, v, p, k, coef, st); break;
+    case 4: launch_update_t<4>(gp, R, n, w, m, v, p, k, coef, st); break;
+    case 8: launch_update_t<8>(gp, R, n, w, m, v, p, k, coef, st); break;
+    default: launch_update_t<0>(gp, R, n, w, m, v, p, k, coef, st); break;
+  }
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  return SLIDEDP_OK;
+}
+
+int ensure_partials(slidedp_ctx* ctx, int64_t need, cudaStream_t st) {
+  if (need <= ctx->partials_cap) return SLIDEDP_OK;
+  // Rare: a step of more than 17 G parameters. Growing keeps the tiles already written.
+  int64_t cap = ctx->partials_cap;
+  while (cap < need) cap *= 2;
+  double* bigger = nullptr;
+  CU(cudaMalloc(&bigger, (size_t)cap * sizeof(double)));
+  cudaError_t e = cudaMemcpyAsync(bigger, ctx->partials, (size_t)ctx->partials_used * sizeof(double),
+                                  cudaMemcpyDeviceToDevice, st);
+  if (e == cudaSuccess) {
+    int rc = bounded_stream_wait(ctx, st, kWaitSeconds);
+    if (rc != SLIDEDP_OK) { cudaFree(bigger); return rc; }
+  } else {
+    cudaFree(bigger);
+    return cuda_fail(ctx, e);
+  }
+  cudaFree(ctx->partials);
+  ctx->partials = bigger;
+  ctx->partials_cap = cap;
+  return SLIDEDP_OK;
+}
+
+int norm_chunk(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, double inv_R,
+               int first_chunk, cudaStream_t st) {
+  if (first_chunk) ctx->partials_used = 0;
+  if (n == 0) return SLIDEDP_OK;
+  const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
+  int rc = ensure_partials(ctx, ctx->partials_used + ntiles, st);
+  if (rc != SLIDEDP_OK) return rc;
+  int sms = 148;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
+  const int64_t max_blocks = (int64_t)sms * 8;
+  const unsigned blocks = (unsigned)(ntiles < max_blocks ? ntiles : max_blocks);
+  double* dst = ctx->partials + ctx->partials_used;
+  const float inv = (float)inv_R;
+  switch (R) {
+    case 1: grad_sumsq_tiles_kernel<1><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, dst); break;
+    case 2: grad_sumsq_tiles_kernel<2><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, dst); break;
+    case 4: grad_sumsq_tiles_kernel<4><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, dst); break;
+    case 8: grad_sumsq_tiles_kernel<8><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, dst); break;
+    default: grad_sumsq_tiles_kernel<0><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, dst); break;
+  }
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  ctx->partials_used += ntiles;
+  return SLIDEDP_OK;
+}
+
+int norm_finish(slidedp_ctx* ctx, double max_norm, cudaStream_t st) {
+  grad_norm_finish_kernel<<<1, kFinishThreads, 0, st>>>(ctx->partials, ctx->partials_used,
+                                                        max_norm, ctx->scalars);
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  ctx->norm_issued = true;
+  return SLIDEDP_OK;
+}
+
+// Copies the four scalars to the pinned mirror on `st` and waits (bounded) for them.
+int fetch_scalars(slidedp_ctx* ctx, cudaStream_t st) {
+  CU(cudaMemcpyAsync(ctx->host_scalars, ctx->scalars, 4 * sizeof(double),
+                     cudaMemcpyDeviceToHost, st));
+  CU(cudaEventRecord(ctx->scalar_event, st));
+  return bounded_event_wait(ctx, ctx->scalar_event, kWaitSeconds);
+}
+
+int is_pinned(slidedp_ctx* ctx, const void* p, bool* pinned) {
+  cudaPointerAttributes a;
+  cudaError_t e = cudaPointerGetAttributes(&a, p);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    *pinned = false;
+    if (e == cudaErrorInvalidValue) return SLIDEDP_OK;  // plain pageable memory on old drivers
+    return cuda_fail(ctx, e);
+  }
+  *pinned = (a.type == cudaMemoryTypeHost);
+  return SLIDEDP_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+extern "C" {
+
+const char* slidedp_strerror(int status) {
+  switch (status) {
+    case SLIDEDP_OK: return "ok";
+    case SLIDEDP_ERR_INVALID_ARG: return "invalid argument";
+    case SLIDEDP_ERR_MISALIGNED: return "a base pointer is not 16-byte aligned";
+    case SLIDEDP_ERR_BUDGET: return "streaming slots exceed the GPU memory budget";
+    case SLIDEDP_ERR_NOT_PINNED: return "host state pointer is not page-locked";
+    case SLIDEDP_ERR_CUDA: return "a CUDA call failed";
+    case SLIDEDP_ERR_TIMEOUT: return "a bounded wait expired";
+    case SLIDEDP_ERR_NO_NORM: return "clipping requested before any norm was finished";
+    default: return "unknown status";
+  }
+}
+
+size_t slidedp_state_bytes(int64_t n) {
+  // BF16 parameter + BF16 gradient + FP32 master + FP32 m + FP32 v
+  return n < 0 ? 0 : (size_t)n * (2 + 2 + 4 + 4 + 4);
+}
+
+int slidedp_last_cuda_error(const slidedp_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+int64_t slidedp_kernel_launches(const slidedp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int slidedp_create(slidedp_ctx** out, int device, size_t gpu_budget_bytes) {
+  if (!out) return SLIDEDP_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess) { (void)cudaGetLastError(); return SLIDEDP_ERR_CUDA; }
+  if (device < 0 || device >= count) return SLIDEDP_ERR_INVALID_ARG;
+  DeviceGuard guard(device);
+  if (!guard.ok) return SLIDEDP_ERR_CUDA;
+  slidedp_ctx* ctx = new (std::nothrow) slidedp_ctx();
+  if (!ctx) return SLIDEDP_ERR_INVALID_ARG;
+  ctx->device = device;
+  ctx->budget = gpu_budget_bytes;
+  cudaError_t e = cudaSuccess;
+  auto step = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
+  step(cudaMalloc(&ctx->partials, (size_t)kInitialPartials * sizeof(double)));
+  ctx->partials_cap = kInitialPartials;
+  step(cudaMalloc(&ctx->scalars, 4 * sizeof(double)));
+  step(cudaMallocHost(&ctx->host_scalars, 4 * sizeof(double)));
+  step(cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking));
+  step(cudaStreamCreateWithFlags(&ctx->s_compute, cudaStreamNonBlocking));
+  step(cudaStreamCreateWithFlags(&ctx->s_out, cudaStreamNonBlocking));
+  step(cudaEventCreateWithFlags(&ctx->scalar_event, cudaEventDisableTiming));
+  for (int i = 0; i < 3; ++i) {
+    step(cudaEventCreateWithFlags(&ctx->ev_loaded[i], cudaEventDisableTiming));
+    step(cudaEventCreateWithFlags(&ctx->ev_updated[i], cudaEventDisableTiming));
+    step(cudaEventCreateWithFlags(&ctx->ev_free[i], cudaEventDisableTiming));
+  }
+  step(cudaEventCreate(&ctx->ev_begin));
+  step(cudaEventCreate(&ctx->ev_norm_done));
+  step(cudaEventCreate(&ctx->ev_end));
+  if (e == cudaSuccess) {
+    const double init[4] = {0.0, 0.0, 1.0, 0.0};
+    step(cudaMemcpy(ctx->scalars, init, sizeof init, cudaMemcpyHostToDevice));
+  }
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    slidedp_destroy(ctx);
+    return SLIDEDP_ERR_CUDA;
+  }
+  *out = ctx;
+  return SLIDEDP_OK;
+}
+
+int slidedp_destroy(slidedp_ctx* ctx) {
+  if (!ctx) return SLIDEDP_OK;
+  DeviceGuard guard(ctx->device);
+  int rc = SLIDEDP_OK;
+  cudaStream_t own[3] = {ctx->s_in, ctx->s_compute, ctx->s_out};
+  for (cudaStream_t s : own)
+    if (s) {
+      int r = bounded_stream_wait(ctx, s, kWaitSeconds);
+      if (r != SLIDEDP_OK && rc == SLIDEDP_OK) rc = r;
+    }
+  for (cudaStream_t s : own) if (s) cudaStreamDestroy(s);
+  auto kill = [](cudaEvent_t ev) { if (ev) cudaEventDestroy(ev); };
+  kill(ctx->scalar_event); kill(ctx->ev_begin); kill(ctx->ev_norm_done); kill(ctx->ev_end);
+  for (int i = 0; i < 3; ++i) { kill(ctx->ev_loaded[i]); kill(ctx->ev_updated[i]); kill(ctx->ev_free[i]); }
+  for (ChunkEvents& c : ctx->timing) {
+    kill(c.h2d_start); kill(c.h2d_end); kill(c.k_start); kill(c.k_end); kill(c.d2h_start); kill(c.d2h_end);
+  }
+  if (ctx->slots) cudaFree(ctx->slots);
+  if (ctx->partials) cudaFree(ctx->partials);
+  if (ctx->scalars) cudaFree(ctx->scalars);
+  if (ctx->host_scalars) cudaFreeHost(ctx->host_scalars);
+  (void)cudaGetLastError();
+  delete ctx;
+  return rc;
+}
+
+int slidedp_grad_norm(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                      double inv_R, int first_chunk, void* cuda_stream) {
+  if (!ctx || n < 0 || inv_R != inv_R) return SLIDEDP_ERR_INVALID_ARG;
+  GradPtrs gp;
+  int rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  return norm_chunk(ctx, gp, R, n, inv_R, first_chunk, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int slidedp_grad_norm_finish(slidedp_ctx* ctx, double max_norm, double* host_norm,
+                             double* host_coef, void* cuda_stream) {
+  if (!ctx || max_norm != max_norm) return SLIDEDP_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int rc = norm_finish(ctx, max_norm, st);
+  if (rc != SLIDEDP_OK) return rc;
+  if (host_norm || host_coef) {
+    rc = fetch_scalars(ctx, st);
+    if (rc != SLIDEDP_OK) return rc;
+    if (host_norm) *host_norm = ctx->host_scalars[1];
+    if (host_coef) *host_coef = ctx->host_scalars[2];
+  }
+  return SLIDEDP_OK;
+}
+
+int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                               float* master, float* m, float* v, void* param_bf16_out,
+                               const slidedp_hparams* hp, void* cuda_stream) {
+  if (!ctx || n < 0) return SLIDEDP_ERR_INVALID_ARG;
+  int rc = check_hparams(hp);
+  if (rc != SLIDEDP_OK) return rc;
+  GradPtrs gp;
+  rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  if (n > 0 && (!master || !m || !v || !param_bf16_out)) return SLIDEDP_ERR_INVALID_ARG;
+  if (!aligned16(master) || !aligned16(m) || !aligned16(v) || !aligned16(param_bf16_out))
+    return SLIDEDP_ERR_MISALIGNED;
+  const bool clip = hp->max_norm > 0.0;
+  if (clip && !ctx->norm_issued) return SLIDEDP_ERR_NO_NORM;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  return launch_update(ctx, gp, R, n, master, m, v, static_cast<uint16_t*>(param_bf16_out),
+                       make_consts(hp), clip ? ctx->scalars + 2 : nullptr,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n_total,
+                        float* host_master, float* host_m, float* host_v, void* param_bf16_out,
+                        int64_t chunk_elems, int nbuf, int norm_ready,
+                        const slidedp_hparams* hp, slidedp_stats* stats) {
+  if (!ctx || n_total < 0) return SLIDEDP_ERR_INVALID_ARG;
+  int rc = check_hparams(hp);
+  if (rc != SLIDEDP_OK) return rc;
+  GradPtrs gp;
+  rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  if (nbuf < 2 || nbuf > 3 || chunk_elems <= 0 || (chunk_elems % kVec) != 0)
+    return SLIDEDP_ERR_INVALID_ARG;
+  if (n_total > 0 && (!host_master || !host_m || !host_v || !param_bf16_out))
+    return SLIDEDP_ERR_INVALID_ARG;
+  if (!aligned16(host_master) || !aligned16(host_m) || !aligned16(host_v) ||
+      !aligned16(param_bf16_out))
+    return SLIDEDP_ERR_MISALIGNED;
+  const bool clip = hp->max_norm > 0.0;
+  if (clip && norm_ready && !ctx->norm_issued) return SLIDEDP_ERR_NO_NORM;
+  if (stats) {
+    memset(stats, 0, sizeof *stats);
+    stats->clip_coef = 1.0;
+  }
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  if (n_total > 0) {
+    const float* hs[3] = {host_master, host_m, host_v};
+    for (const float* h : hs) {
+      bool pinned = false;
+      rc = is_pinned(ctx, h, &pinned);
+      if (rc != SLIDEDP_OK) return rc;
+      if (!pinned) return SLIDEDP_ERR_NOT_PINNED;
+    }
+  }
+
+  // slots: nbuf x {master, m, v} x cap floats
+  const int64_t cap = chunk_elems < n_total ? chunk_elems : ((n_total + kVec - 1) / kVec) * kVec;
+  const size_t need = (size_t)nbuf * 3 * (size_t)cap * sizeof(float);
+  if (ctx->budget && need > ctx->budget) return SLIDEDP_ERR_BUDGET;
+  if (need > ctx->slot_bytes) {
+    if (ctx->slots) { CU(cudaFree(ctx->slots)); ctx->slots = nullptr; ctx->slot_bytes = 0; }
+    CU(cudaMalloc(&ctx->slots, need));
+    ctx->slot_bytes = need;
+  }
+  const int64_t nchunks = n_total == 0 ? 0 : (n_total + chunk_elems - 1) / chunk_elems;
+  if (stats) {
+    while ((int64_t)ctx->timing.size() < nchunks) {
+      ChunkEvents c;
+      CU(cudaEventCreate(&c.h2d_start)); CU(cudaEventCreate(&c.h2d_end));
+      CU(cudaEventCreate(&c.k_start));   CU(cudaEventCreate(&c.k_end));
+      CU(cudaEventCreate(&c.d2h_start)); CU(cudaEventCreate(&c.d2h_end));
+      ctx->timing.push_back(c);
+    }
+  }
+
+  CU(cudaEventRecord(ctx->ev_begin, ctx->s_compute));
+  CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_begin, 0));
+  CU(cudaStreamWaitEvent(ctx->s_out, ctx->ev_begin, 0));
+  if (clip && !norm_ready) {
+    rc = norm_chunk(ctx, gp, R, n_total, hp->inv_R, 1, ctx->s_compute);
+    if (rc != SLIDEDP_OK) return rc;
+    rc = norm_finish(ctx, hp->max_norm, ctx->s_compute);
+    if (rc != SLIDEDP_OK) return rc;
+  }
+  CU(cudaEventRecord(ctx->ev_norm_done, ctx->s_compute));
+
+  const UpdateConsts k = make_consts(hp);
+  const double* coef = clip ? ctx->scalars + 2 : nullptr;
+  uint16_t* pout = static_cast<uint16_t*>(param_bf16_out);
+  for (int64_t c = 0; c < nchunks; ++c) {
+    const int slot = (int)(c % nbuf);
+    const int64_t off = c * chunk_elems;
+    const int64_t len = n_total - off < chunk_elems ? n_total - off : chunk_elems;
+    const size_t bytes = (size_t)len * sizeof(float);
+    float* sw = ctx->slots + (size_t)slot * 3 * cap;
+    float* sm = sw + cap;
+    float* sv = sm + cap;
+    ChunkEvents* te = stats ? &ctx->timing[c] : nullptr;
+    // copy-in: the slot must have been drained by the copy-out of chunk c - nbuf
+    if (c >= nbuf) CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_free[slot], 0));
+    if (te) CU(cudaEventRecord(te->h2d_start, ctx->s_in));
+    CU(cudaMemcpyAsync(sw, host_master + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
+    CU(cudaMemcpyAsync(sm, host_m + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
+    CU(cudaMemcpyAsync(sv, host_v + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
+    if (te) CU(cudaEventRecord(te->h2d_end, ctx->s_in));
+    CU(cudaEventRecord(ctx->ev_loaded[slot], ctx->s_in));
+    // update
+    CU(cudaStreamWaitEvent(ctx->s_compute, ctx->ev_loaded[slot], 0));
+    if (te) CU(cudaEventRecord(te->k_start, ctx->s_compute));
+    GradPtrs gc = gp;
+    for (int r = 0; r < R; ++r) gc.p[r] = gp.p[r] + off;
+    rc = launch_update(ctx, gc, R, len, sw, sm, sv, pout + off, k, coef, ctx->s_compute);
+    if (rc != SLIDEDP_OK) return rc;
+    if (te) CU(cudaEventRecord(te->k_end, ctx->s_compute));
+    CU(cudaEventRecord(ctx->ev_updated[slot], ctx->s_compute));
+    // copy-out
+    CU(cudaStreamWaitEvent(ctx->s_out, ctx->ev_updated[slot], 0));
+    if (te) CU(cudaEventRecord(te->d2h_start, ctx->s_out));
+    CU(cudaMemcpyAsync(host_master + off, sw, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
+    CU(cudaMemcpyAsync(host_m + off, sm, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
+    CU(cudaMemcpyAsync(host_v + off, sv, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
+    if (te) CU(cudaEventRecord(te->d2h_end, ctx->s_out));
+    CU(cudaEventRecord(ctx->ev_free[slot], ctx->s_out));
+  }
+  // the step ends when the compute stream (norm, even with no chunks) and the last
+  // copy-out are both done
+  CU(cudaStreamWaitEvent(ctx->s_out, ctx->ev_norm_done, 0));
+  if (clip) CU(cudaMemcpyAsync(ctx->host_scalars, ctx->scalars, 4 * sizeof(double),
+                               cudaMemcpyDeviceToHost, ctx->s_out));
+  CU(cudaEventRecord(ctx->ev_end, ctx->s_out));
+  rc = bounded_event_wait(ctx, ctx->ev_end, kWaitSeconds);
+  if (rc != SLIDEDP_OK) return rc;
+  rc = bounded_stream_wait(ctx, ctx->s_compute, kWaitSeconds);
+  if (rc != SLIDEDP_OK) return rc;
+  rc = bounded_stream_wait(ctx, ctx->s_in, kWaitSeconds);
+  if (rc != SLIDEDP_OK) return rc;
+
+  if (stats) {
+    float ms = 0.f;
+    CU(cudaEventElapsedTime(&ms, ctx->ev_begin, ctx->ev_end));
+    stats->ms_total = ms;
+    CU(cudaEventElapsedTime(&ms, ctx->ev_begin, ctx->ev_norm_done));
+    stats->ms_norm = (clip && !norm_ready) ? ms : 0.0;
+    stats->chunks = nchunks;
+    for (int64_t c = 0; c < nchunks; ++c) {
+      const ChunkEvents& te = ctx->timing[c];
+      CU(cudaEventElapsedTime(&ms, te.h2d_start, te.h2d_end)); stats->ms_h2d += ms;
+      CU(cudaEventElapsedTime(&ms, te.k_start, te.k_end));     stats->ms_kernel += ms;
+      CU(cudaEventElapsedTime(&ms, te.d2h_start, te.d2h_end)); stats->ms_d2h += ms;
+    }
+    const double link_bytes = 12.0 * (double)n_total;
+    if (stats->ms_h2d > 0) stats->gbs_h2d = link_bytes / (stats->ms_h2d * 1e6);
+    if (stats->ms_d2h > 0) stats->gbs_d2h = link_bytes / (stats->ms_d2h * 1e6);
+    if (clip) {
+      stats->norm = ctx->host_scalars[1];
+      stats->clip_coef = ctx->host_scalars[2];
+      stats->nonfinite = ctx->host_scalars[3] != 0.0;
+    }
+  }
+  return SLIDEDP_OK;
+}
+
+int slidedp_link_probe(slidedp_ctx* ctx, void* host_a, void* host_b, void* dev_a, void* dev_b,
+                       size_t bytes, size_t copy_bytes, int reps, double out4[4]) {
+  if (!ctx || !host_a || !host_b || !dev_a || !dev_b || !out4 || bytes == 0 || copy_bytes == 0 ||
+      reps < 1)
+    return SLIDEDP_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  for (void* h : {host_a, host_b}) {
+    bool pinned = false;
+    int rc = is_pinned(ctx, h, &pinned);
+    if (rc != SLIDEDP_OK) return rc;
+    if (!pinned) return SLIDEDP_ERR_NOT_PINNED;
+  }
+  cudaEvent_t a0, a1, b0, b1;
+  CU(cudaEventCreate(&a0)); CU(cudaEventCreate(&a1)); CU(cudaEventCreate(&b0)); CU(cudaEventCreate(&b1));
+  int rc = SLIDEDP_OK;
+  auto pieces = [&](bool h2d, cudaStream_t st) -> cudaError_t {
+    for (size_t off = 0; off < bytes; off += copy_bytes) {
+      const size_t len = bytes - off < copy_bytes ? bytes - off : copy_bytes;
+      cudaError_t e = h2d ? cudaMemcpyAsync((char*)dev_a + off, (char*)host_a + off, len,
+                                            cudaMemcpyHostToDevice, st)
+                          : cudaMemcpyAsync((char*)host_b + off, (char*)dev_b + off, len,
+                                            cudaMemcpyDeviceToHost, st);
+      if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+  };
+  // mode 0: H2D alone; 1: D2H alone; 2: both at once
+  for (int mode = 0; mode < 3 && rc == SLIDEDP_OK; ++mode) {
+    double best_in = 0.0, best_out = 0.0;
+    for (int rep = 0; rep < reps + 1 && rc == SLIDEDP_OK; ++rep) {  // first pass warms up
+      cudaError_t e = cudaSuccess;
+      if (mode != 1) {
+        e = cudaEventRecord(a0, ctx->s_in);
+        if (e == cudaSuccess) e = pieces(true, ctx->s_in);
+        if (e == cudaSuccess) e = cudaEventRecord(a1, ctx->s_in);
+      }
+      if (e == cudaSuccess && mode != 0) {
+        e = cudaEventRecord(b0, ctx->s_out);
+        if (e == cudaSuccess) e = pieces(false, ctx->s_out);
+        if (e == cudaSuccess) e = cudaEventRecord(b1, ctx->s_out);
+      }
+      if (e != cudaSuccess) { rc = cuda_fail(ctx, e); break; }
+      if (mode != 1) rc = bounded_event_wait(ctx, a1, kWaitSeconds);
+      if (rc == SLIDEDP_OK && mode != 0) rc = bounded_event_wait(ctx, b1, kWaitSeconds);
+      if (rc != SLIDEDP_OK) break;
+      float ms = 0.f;
+      if (mode != 1 && cudaEventElapsedTime(&ms, a0, a1) == cudaSuccess && rep > 0 && ms > 0) {
+        const double g = (double)bytes / (ms * 1e6);
+        if (g > best_in) best_in = g;
+      }
+      if (mode != 0 && cudaEventElapsedTime(&ms, b0, b1) == cudaSuccess && rep > 0 && ms > 0) {
+        const double g = (double)bytes / (ms * 1e6);
+        if (g > best_out) best_out = g;
+      }
+    }
+    if (mode == 0) out4[0] = best_in;
+    if (mode == 1) out4[1] = best_out;
+    if (mode == 2) { out4[2] = best_in; out4[3] = best_out; }
+  }
+  cudaEventDestroy(a0); cudaEventDestroy(a1); cudaEventDestroy(b0); cudaEventDestroy(b1);
+  return rc;
+}
+
+}  // extern "C"

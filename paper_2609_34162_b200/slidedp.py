@@ -1,0 +1,217 @@
+"""Thin ctypes binding over libslidedp (same names as the C ABI in ``include/slidedp.h``).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.
+Tensors are torch tensors used purely as device / pinned-host memory; their
+``data_ptr()`` and the raw ``cudaStream_t`` are what crosses the boundary. There is no CPU
+fallback: if the shared library is missing the import of this module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libslidedp.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2609_34162_b200.build` "
+        "(nvcc, sm_100a). libslidedp has no CPU fallback.")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+MAX_RANKS = 16
+OK, ERR_INVALID_ARG, ERR_MISALIGNED, ERR_BUDGET, ERR_NOT_PINNED, ERR_CUDA, ERR_TIMEOUT, ERR_NO_NORM = (
+    0, -1, -2, -3, -4, -5, -6, -7)
+
+
+class _HParams(ctypes.Structure):
+    _fields_ = [("lr", ctypes.c_double), ("beta1", ctypes.c_double), ("beta2", ctypes.c_double),
+                ("eps", ctypes.c_double), ("weight_decay", ctypes.c_double),
+                ("inv_R", ctypes.c_double), ("max_norm", ctypes.c_double),
+                ("step", ctypes.c_int64)]
+
+
+class _Stats(ctypes.Structure):
+    _fields_ = [("norm", ctypes.c_double), ("clip_coef", ctypes.c_double),
+                ("ms_total", ctypes.c_double), ("ms_norm", ctypes.c_double),
+                ("ms_h2d", ctypes.c_double), ("ms_kernel", ctypes.c_double),
+                ("ms_d2h", ctypes.c_double), ("gbs_h2d", ctypes.c_double),
+                ("gbs_d2h", ctypes.c_double), ("chunks", ctypes.c_int64),
+                ("nonfinite", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+@dataclass
+class HParams:
+    lr: float = 1e-5
+    beta1: float = 0.9
+    beta2: float = 0.95
+    eps: float = 1e-8
+    weight_decay: float = 0.1
+    inv_R: float = 1.0
+    max_norm: float = 0.0
+    step: int = 1
+
+    def _c(self) -> _HParams:
+        return _HParams(self.lr, self.beta1, self.beta2, self.eps, self.weight_decay,
+                        self.inv_R, self.max_norm, int(self.step))
+
+
+_vp, _pp = ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p)
+_lib.slidedp_create.restype = ctypes.c_int
+_lib.slidedp_create.argtypes = [ctypes.POINTER(_vp), ctypes.c_int, ctypes.c_size_t]
+_lib.slidedp_destroy.restype = ctypes.c_int
+_lib.slidedp_destroy.argtypes = [_vp]
+_lib.slidedp_strerror.restype = ctypes.c_char_p
+_lib.slidedp_strerror.argtypes = [ctypes.c_int]
+_lib.slidedp_last_cuda_error.restype = ctypes.c_int
+_lib.slidedp_last_cuda_error.argtypes = [_vp]
+_lib.slidedp_state_bytes.restype = ctypes.c_size_t
+_lib.slidedp_state_bytes.argtypes = [ctypes.c_int64]
+_lib.slidedp_grad_norm.restype = ctypes.c_int
+_lib.slidedp_grad_norm.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, ctypes.c_double,
+                                   ctypes.c_int, _vp]
+_lib.slidedp_grad_norm_finish.restype = ctypes.c_int
+_lib.slidedp_grad_norm_finish.argtypes = [_vp, ctypes.c_double, ctypes.POINTER(ctypes.c_double),
+                                          ctypes.POINTER(ctypes.c_double), _vp]
+_lib.slidedp_reduce_adamw_chunk.restype = ctypes.c_int
+_lib.slidedp_reduce_adamw_chunk.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp,
+                                            _vp, ctypes.POINTER(_HParams), _vp]
+_lib.slidedp_stream_step.restype = ctypes.c_int
+_lib.slidedp_stream_step.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp, _vp,
+                                     ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                     ctypes.POINTER(_HParams), ctypes.POINTER(_Stats)]
+_lib.slidedp_link_probe.restype = ctypes.c_int
+_lib.slidedp_link_probe.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, ctypes.c_size_t,
+                                    ctypes.c_int, ctypes.POINTER(ctypes.c_double)]
+_lib.slidedp_kernel_launches.restype = ctypes.c_int64
+_lib.slidedp_kernel_launches.argtypes = [_vp]
+
+
+class SlideDPError(RuntimeError):
+    def __init__(self, status: int, cuda_error: int = 0):
+        self.status, self.cuda_error = status, cuda_error
+        msg = _lib.slidedp_strerror(status).decode()
+        if status == ERR_CUDA:
+            msg += f" (cudaError_t {cuda_error})"
+        super().__init__(f"libslidedp: {msg} [{status}]")
+
+
+def slidedp_strerror(status: int) -> str:
+    return _lib.slidedp_strerror(status).decode()
+
+
+def slidedp_state_bytes(n: int) -> int:
+    return int(_lib.slidedp_state_bytes(n))
+
+
+def _ptr(x) -> int:
+    """Raw address of a tensor's first element (or an int passed through, or None)."""
+    if x is None:
+        return 0
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()
+
+
+def _grad_array(grads):
+    return (ctypes.c_void_p * len(grads))(*[_ptr(g) for g in grads])
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+class Context:
+    """Owns a ``slidedp_ctx``. Methods carry the C entry points' names and argument order."""
+
+    def __init__(self, device: int = 0, gpu_budget_bytes: int = 0):
+        self._h = _vp()
+        rc = _lib.slidedp_create(ctypes.byref(self._h), device, gpu_budget_bytes)
+        if rc != OK:
+            self._h = _vp()
+            raise SlideDPError(rc)
+        self.device = device
+
+    def _check(self, rc: int):
+        if rc != OK:
+            raise SlideDPError(rc, _lib.slidedp_last_cuda_error(self._h))
+
+    def slidedp_destroy(self):
+        if self._h:
+            rc = _lib.slidedp_destroy(self._h)
+            self._h = _vp()
+            if rc != OK:
+                raise SlideDPError(rc)
+
+    close = slidedp_destroy
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.slidedp_destroy()
+
+    def __del__(self):
+        try:
+            if self._h:
+                _lib.slidedp_destroy(self._h)
+                self._h = _vp()
+        except Exception:
+            pass
+
+    def slidedp_kernel_launches(self) -> int:
+        return int(_lib.slidedp_kernel_launches(self._h))
+
+    def slidedp_grad_norm(self, grads, n: int, inv_R: float, first_chunk: bool = True,
+                          stream=None) -> None:
+        self._check(_lib.slidedp_grad_norm(self._h, _grad_array(grads), len(grads), n, inv_R,
+                                           int(first_chunk), _stream(stream)))
+
+    def slidedp_grad_norm_finish(self, max_norm: float, fetch: bool = False, stream=None):
+        """Returns (norm, coef) if ``fetch`` (synchronises), else None."""
+        if fetch:
+            norm, coef = ctypes.c_double(), ctypes.c_double()
+            self._check(_lib.slidedp_grad_norm_finish(self._h, max_norm, ctypes.byref(norm),
+                                                      ctypes.byref(coef), _stream(stream)))
+            return norm.value, coef.value
+        self._check(_lib.slidedp_grad_norm_finish(self._h, max_norm, None, None, _stream(stream)))
+        return None
+
+    def slidedp_reduce_adamw_chunk(self, grads, n: int, master, m, v, param_bf16_out,
+                                   hp: HParams, stream=None) -> None:
+        c = hp._c()
+        self._check(_lib.slidedp_reduce_adamw_chunk(
+            self._h, _grad_array(grads), len(grads), n, _ptr(master), _ptr(m), _ptr(v),
+            _ptr(param_bf16_out), ctypes.byref(c), _stream(stream)))
+
+    def slidedp_stream_step(self, grads, n_total: int, host_master, host_m, host_v,
+                            param_bf16_out, chunk_elems: int, nbuf: int, hp: HParams,
+                            norm_ready: bool = False, want_stats: bool = True):
+        c = hp._c()
+        st = _Stats()
+        self._check(_lib.slidedp_stream_step(
+            self._h, _grad_array(grads), len(grads), n_total, _ptr(host_master), _ptr(host_m),
+            _ptr(host_v), _ptr(param_bf16_out), chunk_elems, nbuf, int(norm_ready),
+            ctypes.byref(c), ctypes.byref(st) if want_stats else None))
+        if not want_stats:
+            return None
+        return {f: getattr(st, f) for f, _ in _Stats._fields_ if f != "reserved"}
+
+    def slidedp_link_probe(self, host_a, host_b, dev_a, dev_b, nbytes: int, copy_bytes: int,
+                           reps: int = 3):
+        out = (ctypes.c_double * 4)()
+        self._check(_lib.slidedp_link_probe(self._h, _ptr(host_a), _ptr(host_b), _ptr(dev_a),
+                                            _ptr(dev_b), nbytes, copy_bytes, reps, out))
+        return {"h2d": out[0], "d2h": out[1], "h2d_bidir": out[2], "d2h_bidir": out[3]}
+
+
+def slidedp_create(device: int = 0, gpu_budget_bytes: int = 0) -> Context:
+    return Context(device, gpu_budget_bytes)

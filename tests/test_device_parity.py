@@ -1,0 +1,253 @@
+"""GPU parity, device-resident mode: libslidedp (through its C ABI) against the CPU oracle,
+element by element, on the same seeded inputs."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity
+from paper_2609_34162_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+NTHREADS = max(1, min(64, len(os.sched_getaffinity(0))))
+
+
+@pytest.fixture(scope="module")
+def sd():
+    import paper_2609_34162_b200.slidedp as sd
+    return sd
+
+
+@pytest.fixture()
+def ctx(sd):
+    c = sd.slidedp_create(0, 0)
+    yield c
+    c.slidedp_destroy()
+
+
+def hp_pair(sd, **kw):
+    return sd.HParams(**kw), oracle.HParams(**kw)
+
+
+def random_case(n, R, seed, zero_moments=False, sigma=1e-3):
+    g = torch.Generator().manual_seed(seed)
+    grads = [(torch.randn(n, generator=g) * sigma).to(torch.bfloat16) for _ in range(R)]
+    w = torch.randn(n, generator=g) * 0.02
+    if zero_moments:
+        m, v = torch.zeros(n), torch.zeros(n)
+    else:
+        m = torch.randn(n, generator=g) * 3e-4
+        v = torch.randn(n, generator=g).square() * 1e-7
+    return grads, w, m, v
+
+
+def run_both(ctx, sd, grads, w, m, v, hp_kw, clip, chunk=None):
+    """One step on the GPU (C ABI) and in the oracle; returns both results on the host."""
+    n, R = w.numel(), len(grads)
+    hp_g, hp_o = hp_pair(sd, inv_R=1.0 / R, max_norm=clip, **hp_kw)
+    dg = [g.cuda() for g in grads]
+    dw, dm, dv = w.cuda(), m.cuda(), v.cuda()
+    dp = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    norm_g = None
+    if clip > 0:
+        ctx.slidedp_grad_norm(dg, n, hp_g.inv_R, True)
+        norm_g, coef_g = ctx.slidedp_grad_norm_finish(clip, fetch=True)
+    if chunk is None:
+        ctx.slidedp_reduce_adamw_chunk(dg, n, dw, dm, dv, dp, hp_g)
+    else:
+        for lo in range(0, n, chunk):
+            k = min(chunk, n - lo)
+            ctx.slidedp_reduce_adamw_chunk([g[lo:] for g in dg], k, dw[lo:], dm[lo:], dv[lo:],
+                                           dp[lo:], hp_g)
+    torch.cuda.synchronize()
+    ow, om, ov = parity.f32(w).copy(), parity.f32(m).copy(), parity.f32(v).copy()
+    op = np.zeros(n, np.uint16)
+    norm_o, coef_o = oracle.step([parity.u16(g) for g in grads], ow, om, ov, op, hp_o,
+                                 nthreads=NTHREADS)
+    return (parity.f32(dw), parity.f32(dm), parity.f32(dv), parity.u16(dp), norm_g), \
+           (ow, om, ov, op, norm_o)
+
+
+def assert_parity(tag, got, want, clip):
+    for name, a, b in zip(("master", "m", "v"), got[:3], want[:3]):
+        parity.assert_fp32_close(f"{tag}/{name}", a, b)
+    parity.assert_bf16_close(f"{tag}/param_bf16", got[3], want[3])
+    if clip > 0:
+        parity.assert_norm_close(got[4], want[4])
+
+
+ADAM = dict(lr=1e-5, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
+
+
+@pytest.mark.parametrize("R", [1, 2, 3, 4, 5, 8, 16])
+@pytest.mark.parametrize("n", [1, 7, 8, 9, 1023, 2048 * 3 + 5, (1 << 20) + 3])
+def test_odd_sizes_all_rank_counts(ctx, sd, n, R):
+    grads, w, m, v = random_case(n, R, seed=1000 * R + n % 997)
+    for clip, step in ((0.0, 1), (0.05, 11)):
+        got, want = run_both(ctx, sd, grads, w, m, v, dict(ADAM, step=step), clip)
+        assert_parity(f"n={n} R={R} clip={clip}", got, want, clip)
+
+
+def test_empty_chunk_is_a_no_op(ctx, sd):
+    hp_g, _ = hp_pair(sd, inv_R=0.5, step=1, **ADAM)
+    g = [torch.zeros(8, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    w = torch.ones(8, device="cuda")
+    p = torch.zeros(8, dtype=torch.bfloat16, device="cuda")
+    before = ctx.slidedp_kernel_launches()
+    ctx.slidedp_reduce_adamw_chunk(g, 0, w, w.clone(), w.clone(), p, hp_g)
+    ctx.slidedp_grad_norm(g, 0, 0.5, True)
+    norm, coef = ctx.slidedp_grad_norm_finish(1.0, fetch=True)
+    assert (norm, coef) == (0.0, 1.0) and torch.all(w == 1.0)
+    assert ctx.slidedp_kernel_launches() == before + 1          # only the finish kernel ran
+
+
+def test_config1_tiny_chunk_first_step(ctx, sd):
+    """One flat chunk of 2^20 parameters, R = 2, zero moments, step 1, no clipping."""
+    wl = W.CONFIGS["tiny"]
+    grads = [W.rank_gradient(wl, r, step=1) for r in range(wl.R)]
+    w = W.master_weights(wl)
+    z = torch.zeros(wl.numel)
+    got, want = run_both(ctx, sd, grads, w, z, z.clone(), dict(wl.hparams, step=1), 0.0)
+    assert_parity("tiny", got, want, 0.0)
+
+
+def prewarmed_state(wl, device="cpu"):
+    """m, v (and the master) after `prewarm_steps` seeded ORACLE steps; never the CUDA path."""
+    w = parity.f32(W.master_weights(wl, device=device)).copy()
+    n = w.size
+    m, v, p = np.zeros(n, np.float32), np.zeros(n, np.float32), np.zeros(n, np.uint16)
+    for t in range(1, wl.prewarm_steps + 1):
+        grads = [parity.u16(W.rank_gradient(wl, r, step=t, device=device)) for r in range(wl.R)]
+        hp = oracle.HParams(inv_R=1.0 / wl.R, max_norm=wl.max_norm, step=t, **wl.hparams)
+        oracle.step(grads, w, m, v, p, hp, nthreads=NTHREADS)
+    return w, m, v
+
+
+@pytest.mark.parametrize("divisor", [16, 1])
+def test_config2_qwen3_8b_layer_step11_clipped(ctx, sd, divisor):
+    """Qwen3-8B-shaped layer, R = 4, moments pre-warmed by 10 seeded steps, step 11, clip 1.0.
+    divisor 1 is the full 192,946,176-parameter layer, compared element by element."""
+    wl = W.CONFIGS["qwen3_8b_layer"]
+    if divisor > 1:
+        wl = W.scaled(wl, divisor)
+    dev = "cuda"      # draw on the GPU (fast at full size); both sides get the same bits
+    w, m, v = prewarmed_state(wl, dev)
+    t = wl.first_step
+    grads = [W.rank_gradient(wl, r, step=t, device=dev).cpu() for r in range(wl.R)]
+    got, want = run_both(ctx, sd, grads, torch.from_numpy(w), torch.from_numpy(m),
+                         torch.from_numpy(v), dict(wl.hparams, step=t), wl.max_norm)
+    assert want[4] > 2.0, "clipping must be active in this configuration"
+    assert_parity(wl.name, got, want, wl.max_norm)
+
+
+def test_norm_is_deterministic_and_chunk_invariant(ctx, sd):
+    n, R = 16384 * 37 + 4321, 4
+    grads, *_ = random_case(n, R, seed=77, sigma=1e-2)
+    dg = [g.cuda() for g in grads]
+    ref = None
+    for _ in range(3):
+        ctx.slidedp_grad_norm(dg, n, 0.25, True)
+        out = ctx.slidedp_grad_norm_finish(1.0, fetch=True)
+        ref = ref or out
+        assert out == ref                                        # bit-identical run to run
+    # chunks cut at multiples of the 16384-element tile: bit-identical to the uncut pass
+    for cut in (16384, 16384 * 5, 16384 * 36):
+        first = True
+        for lo in range(0, n, cut):
+            ctx.slidedp_grad_norm([g[lo:] for g in dg], min(cut, n - lo), 0.25, first)
+            first = False
+        assert ctx.slidedp_grad_norm_finish(1.0, fetch=True) == ref
+    # any other cut: same value to rounding
+    first = True
+    for lo in range(0, n, 100_000):
+        ctx.slidedp_grad_norm([g[lo:] for g in dg], min(100_000, n - lo), 0.25, first)
+        first = False
+    other = ctx.slidedp_grad_norm_finish(1.0, fetch=True)
+    assert abs(other[0] - ref[0]) <= 1e-12 * ref[0]
+    want = oracle.clip_coef(oracle.grad_sumsq([parity.u16(g) for g in grads], 0.25), 1.0)
+    parity.assert_norm_close(ref[0], want[1])
+    assert abs(ref[1] - want[0]) <= 1e-6 * want[0]
+
+
+def test_update_is_chunk_invariant_bit_for_bit(ctx, sd):
+    n, R = (1 << 18) + 8 * 13, 4
+    grads, w, m, v = random_case(n, R, seed=5)
+    whole, want = run_both(ctx, sd, grads, w, m, v, dict(ADAM, step=3), 0.02)
+    assert_parity("whole", whole, want, 0.02)
+    for chunk in (8, 4096, 100_000 - 100_000 % 8):
+        parts, _ = run_both(ctx, sd, grads, w, m, v, dict(ADAM, step=3), 0.02, chunk=chunk)
+        for a, b in zip(whole[:4], parts[:4]):
+            assert np.array_equal(a, b)
+
+
+def test_hyperparameter_and_value_ranges(ctx, sd):
+    """Large lr, tiny and zero gradients, zero state, huge v, denormal-range gradients."""
+    n, R = 4096 + 3, 2
+    g = torch.Generator().manual_seed(9)
+    mag = 10.0 ** (torch.rand(n, generator=g) * 36 - 34)          # 1e-34 .. 1e2
+    sign = torch.where(torch.rand(n, generator=g) < 0.5, -1.0, 1.0)
+    grads = [(mag * sign).to(torch.bfloat16), (mag * 0.5).to(torch.bfloat16)]
+    grads[0][:16] = 0; grads[1][:16] = 0
+    w = torch.randn(n, generator=g) * 0.02
+    w[:4] = 0
+    m = torch.zeros(n); v = torch.zeros(n)
+    m[100:200] = torch.randn(100, generator=g) * 1e-20
+    v[200:300] = 1e30
+    for kw in (dict(lr=1e-2, beta1=0.5, beta2=0.999, eps=1e-6, weight_decay=0.0, step=2),
+               dict(lr=1e-5, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1, step=100000),
+               dict(lr=3e-4, beta1=0.0, beta2=0.0, eps=1e-8, weight_decay=0.01, step=1)):
+        got, want = run_both(ctx, sd, grads, w, m, v, kw, 0.0)
+        assert not np.isnan(got[0]).any()
+        assert_parity(str(kw), got, want, 0.0)
+
+
+def test_nonfinite_gradients_propagate_without_trapping(ctx, sd):
+    n, R = 64, 2
+    grads, w, m, v = random_case(n, R, seed=3)
+    grads[0][5] = float("inf"); grads[1][9] = float("nan")
+    got, want = run_both(ctx, sd, grads, w, m, v, dict(ADAM, step=2), 0.0)
+    for a, b in zip(got[:3], want[:3]):
+        assert np.array_equal(np.isfinite(a), np.isfinite(b))
+    keep = np.ones(n, bool); keep[[5, 9]] = False
+    for a, b in zip(got[:3], want[:3]):
+        parity.assert_fp32_close("finite part", a[keep], b[keep])
+    dg = [g.cuda() for g in grads]
+    ctx.slidedp_grad_norm(dg, n, 0.5, True)
+    norm, coef = ctx.slidedp_grad_norm_finish(1.0, fetch=True)
+    assert np.isnan(norm) and np.isnan(coef)
+
+
+def test_argument_errors_are_reported_not_faulted(ctx, sd):
+    n = 64
+    g = [torch.zeros(n + 8, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    w = torch.zeros(n + 8, device="cuda")
+    p = torch.zeros(n + 8, dtype=torch.bfloat16, device="cuda")
+    hp = sd.HParams(inv_R=0.5, step=1)
+
+    def status(fn):
+        with pytest.raises(sd.SlideDPError) as e:
+            fn()
+        return e.value.status
+
+    call = ctx.slidedp_reduce_adamw_chunk
+    assert status(lambda: call([g[0][1:], g[1]], n, w, w.clone(), w.clone(), p, hp)) == sd.ERR_MISALIGNED
+    assert status(lambda: call(g, n, w[1:], w.clone(), w.clone(), p, hp)) == sd.ERR_MISALIGNED
+    assert status(lambda: call(g, -1, w, w.clone(), w.clone(), p, hp)) == sd.ERR_INVALID_ARG
+    assert status(lambda: call([], n, w, w.clone(), w.clone(), p, hp)) == sd.ERR_INVALID_ARG
+    assert status(lambda: call(g * 9, n, w, w.clone(), w.clone(), p, hp)) == sd.ERR_INVALID_ARG
+    assert status(lambda: call(g, n, None, w.clone(), w.clone(), p, hp)) == sd.ERR_INVALID_ARG
+    assert status(lambda: call(g, n, w, w.clone(), w.clone(), p,
+                               sd.HParams(inv_R=0.5, step=0))) == sd.ERR_INVALID_ARG
+    assert status(lambda: call(g, n, w, w.clone(), w.clone(), p,
+                               sd.HParams(inv_R=0.5, beta1=1.0))) == sd.ERR_INVALID_ARG
+    fresh = sd.slidedp_create(0, 0)
+    try:
+        assert status(lambda: fresh.slidedp_reduce_adamw_chunk(
+            g, n, w, w.clone(), w.clone(), p, sd.HParams(inv_R=0.5, max_norm=1.0))) == sd.ERR_NO_NORM
+    finally:
+        fresh.slidedp_destroy()
+    torch.cuda.synchronize()
+    assert torch.all(w == 0)

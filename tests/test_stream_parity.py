@@ -1,0 +1,195 @@
+"""GPU parity, host-resident mode: FP32 state in pinned host memory, streamed through device
+slots by slidedp_stream_step, against the CPU oracle and against the device-resident path."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import parity
+from paper_2609_34162_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+NTHREADS = max(1, min(64, len(os.sched_getaffinity(0))))
+FULL = os.environ.get("SLIDEDP_FULL_PARITY", "0") == "1"
+
+
+@pytest.fixture(scope="module")
+def sd():
+    import paper_2609_34162_b200.slidedp as sd
+    return sd
+
+
+@pytest.fixture()
+def ctx(sd):
+    c = sd.slidedp_create(0, 0)
+    yield c
+    c.slidedp_destroy()
+
+
+def pinned(a: np.ndarray) -> torch.Tensor:
+    t = torch.empty(a.shape, dtype=torch.float32, pin_memory=True)
+    t.numpy()[...] = a
+    return t
+
+
+def prewarmed_state(wl, layer=0):
+    w = parity.f32(W.master_weights(wl, layer=layer, device="cuda")).copy()
+    n = w.size
+    m, v, p = np.zeros(n, np.float32), np.zeros(n, np.float32), np.zeros(n, np.uint16)
+    for t in range(1, wl.prewarm_steps + 1):
+        grads = [parity.u16(W.rank_gradient(wl, r, step=t, layer=layer, device="cuda"))
+                 for r in range(wl.R)]
+        hp = oracle.HParams(inv_R=1.0 / wl.R, max_norm=wl.max_norm, step=t, **wl.hparams)
+        oracle.step(grads, w, m, v, p, hp, nthreads=NTHREADS)
+    return w, m, v
+
+
+def stream_case(ctx, sd, wl, chunk_elems_list, nbuf_list):
+    """Runs the measured step of a single-layer host-resident workload for every
+    (chunk size, nbuf) and checks each against one oracle step."""
+    n, R, t = wl.numel, wl.R, wl.first_step
+    w0, m0, v0 = prewarmed_state(wl)
+    dg = [W.rank_gradient(wl, r, step=t, device="cuda") for r in range(R)]
+    kw = dict(inv_R=1.0 / R, max_norm=wl.max_norm, step=t, **wl.hparams)
+    ow, om, ov, op = w0.copy(), m0.copy(), v0.copy(), np.zeros(n, np.uint16)
+    norm_o, coef_o = oracle.step([parity.u16(g) for g in dg], ow, om, ov, op,
+                                 oracle.HParams(**kw), nthreads=NTHREADS)
+    results = []
+    for ce in chunk_elems_list:
+        for nbuf in nbuf_list:
+            hw, hm, hv = pinned(w0), pinned(m0), pinned(v0)
+            dp = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+            st = ctx.slidedp_stream_step(dg, n, hw, hm, hv, dp, ce, nbuf, sd.HParams(**kw))
+            tag = f"{wl.name} chunk={ce} nbuf={nbuf}"
+            parity.assert_fp32_close(tag + "/master", hw.numpy(), ow)
+            parity.assert_fp32_close(tag + "/m", hm.numpy(), om)
+            parity.assert_fp32_close(tag + "/v", hv.numpy(), ov)
+            parity.assert_bf16_close(tag + "/param_bf16", parity.u16(dp), op)
+            if wl.max_norm > 0:
+                parity.assert_norm_close(st["norm"], norm_o)
+                assert abs(st["clip_coef"] - coef_o) <= 1e-6 * coef_o
+            assert st["chunks"] == -(-n // ce)
+            results.append((hw.numpy().copy(), hm.numpy().copy(), hv.numpy().copy(),
+                            parity.u16(dp).copy()))
+    return results, (dg, w0, m0, v0, kw)
+
+
+def test_config3_scaled_all_slot_counts_and_device_equivalence(ctx, sd):
+    """Qwen3-14B-shaped layer shrunk 16-fold; chunk sizes that leave a short last chunk;
+    2 and 3 slots; and the host-resident result equals the device-resident one bit for bit."""
+    wl = W.scaled(W.CONFIGS["qwen3_14b_layer_host"], 16)
+    results, (dg, w0, m0, v0, kw) = stream_case(ctx, sd, wl, [1 << 20, 3 * (1 << 19) + 8, 1 << 25],
+                                               [2, 3])
+    for r in results[1:]:
+        for a, b in zip(results[0], r):
+            assert np.array_equal(a, b)                       # chunking / slots never change bits
+    n = wl.numel
+    dw, dm, dv = (torch.from_numpy(x).cuda() for x in (w0, m0, v0))
+    dp = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    ctx.slidedp_grad_norm(dg, n, kw["inv_R"], True)
+    ctx.slidedp_grad_norm_finish(kw["max_norm"])
+    ctx.slidedp_reduce_adamw_chunk(dg, n, dw, dm, dv, dp, sd.HParams(**kw))
+    torch.cuda.synchronize()
+    for a, b in zip(results[0], (parity.f32(dw), parity.f32(dm), parity.f32(dv), parity.u16(dp))):
+        assert np.array_equal(a, b)
+
+
+def test_config3_qwen3_14b_layer_full_size(ctx, sd):
+    """330,311,680 parameters, 64 MiB chunks (16 Mi parameters), triple buffering."""
+    wl = W.CONFIGS["qwen3_14b_layer_host"]
+    stream_case(ctx, sd, wl, [W.chunk_elems(64)], [3])
+
+
+def test_config4_heavy_tailed_chunk_sweep(ctx, sd):
+    """Qwen2.5-72B-shaped layer with 1% Student-t(3) gradients; chunk sizes 16/64/256 MiB.
+    Full size (877,660,160 parameters) with SLIDEDP_FULL_PARITY=1, else shrunk 8-fold."""
+    wl = W.CONFIGS["qwen25_72b_layer_host"]
+    if not FULL:
+        wl = W.scaled(wl, 8)
+    stream_case(ctx, sd, wl, [W.chunk_elems(c) for c in wl.chunk_mib], [3])
+
+
+def test_config5_eight_layers_ten_steps_global_norm(ctx, sd):
+    """Eight Qwen3-14B-shaped layers, R = 8, ten consecutive steps from zero moments; the norm
+    covers all eight layers before any update; BF16 params compared at steps 1, 5 and 10
+    (FP32 state too). Full size with SLIDEDP_FULL_PARITY=1, else shrunk 16-fold."""
+    wl = W.CONFIGS["qwen3_14b_8layers_host"]
+    if not FULL:
+        wl = W.scaled(wl, 16)
+    L, R, nl = wl.layers, wl.R, wl.layer_numel
+    ce = W.chunk_elems(64) if FULL else 1 << 20
+    # GPU side: per-layer pinned state, gradients regenerated per step
+    host = []
+    for l in range(L):
+        w = W.master_weights(wl, layer=l, device="cuda").cpu()
+        host.append([pinned(w.numpy()), pinned(np.zeros(nl, np.float32)),
+                     pinned(np.zeros(nl, np.float32))])
+    ow = [h[0].numpy().copy() for h in host]
+    om = [np.zeros(nl, np.float32) for _ in range(L)]
+    ov = [np.zeros(nl, np.float32) for _ in range(L)]
+    dp = [torch.zeros(nl, dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+    dg = [[torch.empty(nl, dtype=torch.bfloat16, device="cuda") for _ in range(R)] for _ in range(L)]
+    for t in range(1, wl.steps + 1):
+        kw = dict(inv_R=1.0 / R, max_norm=wl.max_norm, step=t, **wl.hparams)
+        S = 0.0
+        for l in range(L):
+            for r in range(R):
+                W.rank_gradient(wl, r, step=t, layer=l, device="cuda", out=dg[l][r])
+            ctx.slidedp_grad_norm(dg[l], nl, kw["inv_R"], l == 0)
+        norm_g, coef_g = ctx.slidedp_grad_norm_finish(wl.max_norm, fetch=True)
+        for l in range(L):
+            ctx.slidedp_stream_step(dg[l], nl, host[l][0], host[l][1], host[l][2], dp[l], ce, 3,
+                                    sd.HParams(**kw), norm_ready=True)
+        # oracle: the same step, norm over all layers first, then every layer
+        hg = [[parity.u16(g) for g in dg[l]] for l in range(L)]
+        for l in range(L):
+            S += oracle.grad_sumsq(hg[l], kw["inv_R"], NTHREADS)
+        coef_o, norm_o = oracle.clip_coef(S, wl.max_norm)
+        parity.assert_norm_close(norm_g, norm_o)
+        assert coef_o < 1.0
+        check = t in (1, 5, 10)
+        for l in range(L):
+            op = np.zeros(nl, np.uint16)
+            oracle.reduce_adamw_chunk(hg[l], ow[l], om[l], ov[l], op, oracle.HParams(**kw),
+                                      clip=coef_o, nthreads=NTHREADS)
+            if check:
+                tag = f"step {t} layer {l}"
+                parity.assert_bf16_close(tag + "/param_bf16", parity.u16(dp[l]), op)
+                parity.assert_fp32_close(tag + "/master", host[l][0].numpy(), ow[l])
+                parity.assert_fp32_close(tag + "/m", host[l][1].numpy(), om[l])
+                parity.assert_fp32_close(tag + "/v", host[l][2].numpy(), ov[l])
+
+
+def test_stream_step_argument_errors(ctx, sd):
+    n = 1 << 12
+    g = [torch.zeros(n, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    p = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    hw, hm, hv = (torch.zeros(n, pin_memory=True) for _ in range(3))
+    pageable = torch.zeros(n)
+    hp = sd.HParams(inv_R=0.5, step=1)
+
+    def status(fn):
+        with pytest.raises(sd.SlideDPError) as e:
+            fn()
+        return e.value.status
+
+    call = ctx.slidedp_stream_step
+    assert status(lambda: call(g, n, pageable, hm, hv, p, 1024, 3, hp)) == sd.ERR_NOT_PINNED
+    assert status(lambda: call(g, n, hw, hm, hv, p, 1024, 4, hp)) == sd.ERR_INVALID_ARG
+    assert status(lambda: call(g, n, hw, hm, hv, p, 1001, 3, hp)) == sd.ERR_INVALID_ARG
+    assert status(lambda: call(g, n, hw, hm, hv, p, 0, 3, hp)) == sd.ERR_INVALID_ARG
+    small = sd.slidedp_create(0, 3 * 3 * 1024 * 4 - 1)            # one byte short of three slots
+    try:
+        assert status(lambda: small.slidedp_stream_step(g, n, hw, hm, hv, p, 1024, 3, hp)) == sd.ERR_BUDGET
+        st = small.slidedp_stream_step(g, n, hw, hm, hv, p, 1024, 2, hp)     # two slots fit
+        assert st["chunks"] == 4
+        assert status(lambda: small.slidedp_stream_step(
+            g, n, hw, hm, hv, p, 1024, 2, sd.HParams(inv_R=0.5, max_norm=1.0),
+            norm_ready=True)) == sd.ERR_NO_NORM
+    finally:
+        small.slidedp_destroy()
+    st = call(g, 0, hw, hm, hv, p, 1024, 3, hp)
+    assert st["chunks"] == 0

@@ -139,7 +139,7 @@ def test_config2_qwen3_8b_layer_step11_clipped(ctx, sd, divisor):
     grads = [W.rank_gradient(wl, r, step=t, device=dev).cpu() for r in range(wl.R)]
     got, want = run_both(ctx, sd, grads, torch.from_numpy(w), torch.from_numpy(m),
                          torch.from_numpy(v), dict(wl.hparams, step=t), wl.max_norm)
-    assert want[4] > 2.0, "clipping must be active in this configuration"
+    assert want[4] > 1.5, "clipping must be active in this configuration"
     assert_parity(wl.name, got, want, wl.max_norm)
 
 

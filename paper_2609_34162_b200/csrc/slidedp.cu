@@ -405,7 +405,7 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
   GradPtrs gp;
   rc = check_grads(grads_bf16, R, &gp);
   if (rc != SLIDEDP_OK) return rc;
-  if (nbuf < 2 || nbuf > 3 || chunk_elems <= 0 || (chunk_elems % kVec) != 0)
+  if (nbuf < 2 || nbuf > 3 || chunk_elems <= 0 || (chunk_elems % 8) != 0)
     return SLIDEDP_ERR_INVALID_ARG;
   if (n_total > 0 && (!host_master || !host_m || !host_v || !param_bf16_out))
     return SLIDEDP_ERR_INVALID_ARG;
@@ -431,7 +431,7 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
   }
 
   // slots: nbuf x {master, m, v} x cap floats
-  const int64_t cap = chunk_elems < n_total ? chunk_elems : ((n_total + kVec - 1) / kVec) * kVec;
+  const int64_t cap = chunk_elems < n_total ? chunk_elems : ((n_total + 7) / 8) * 8;
   const size_t need = (size_t)nbuf * 3 * (size_t)cap * sizeof(float);
   if (ctx->budget && need > ctx->budget) return SLIDEDP_ERR_BUDGET;
   if (need > ctx->slot_bytes) {

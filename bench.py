@@ -33,8 +33,9 @@ WORKLOAD = "qwen3_8b_layer"
 HOST_WORKLOAD = "qwen3_14b_layer_host"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter of the fused update kernel, from
-# the ncu capture summarised in profiles/reduce_adamw_kernel_R4.md (None until captured).
-NCU_TRAFFIC_BYTES_PER_PARAM = None
+# the ncu capture summarised in profiles/reduce_adamw_kernel_R4_50M_params.md (50 M-parameter case,
+# scaled to a full launch by the parameter count).
+NCU_TRAFFIC_BYTES_PER_PARAM = 32.92
 
 
 def measured_peak_hbm():
@@ -313,6 +314,144 @@ def run_cuda(args):
     return 0
 
 
+def run_sweep(args):
+    """`--report sweep`: one JSON line with the other benchmark configurations on one GPU:
+    the tiny chunk (L2-resident and rotating over buffer sets larger than L2), the chunk-size
+    sweep of the Qwen2.5-72B-shaped layer (16/64/256 MiB, 2 and 3 slots) and the eight-layer,
+    R = 8 host-resident step with one global norm. Not the contract line; for the tables."""
+    import torch
+
+    import paper_2609_34162_b200.slidedp as sd
+    from paper_2609_34162_b200 import workloads as W
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    ctx = sd.slidedp_create(0, 0)
+    st = torch.cuda.current_stream()
+    peak, peak_kind = measured_peak_hbm()
+    out = {"report": "sweep", "hbm_peak_gbs": peak, "hbm_peak_source": peak_kind}
+
+    def hp(wl, t):
+        return sd.HParams(inv_R=1.0 / wl.R, max_norm=wl.max_norm, step=t, **wl.hparams)
+
+    # ---- tiny chunk: 31.5 MB of traffic fits the 126 MB L2, so time it both ways
+    wl = W.CONFIGS["tiny"]
+    n, R, sets = wl.numel, wl.R, 16
+    bufs = []
+    for i in range(sets):
+        g = [W.rank_gradient(wl, r, step=1 + i, device=dev) for r in range(R)]
+        bufs.append((g, W.master_weights(wl, device=dev), torch.zeros(n, device=dev),
+                     torch.zeros(n, device=dev), torch.zeros(n, dtype=torch.bfloat16, device=dev)))
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    res = {}
+    reps = sets * 20
+    for name, pick in (("l2_resident", lambda i: 0), ("rotating_16_sets", lambda i: i % sets)):
+        for i in range(sets * 2):
+            g, w, m, v, p = bufs[pick(i)]
+            ctx.slidedp_reduce_adamw_chunk(g, n, w, m, v, p, hp(wl, 1))
+        torch.cuda.synchronize()
+        # a 5 us kernel is launch-bound from Python: capture the launches in a CUDA graph
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(reps):
+                g, w, m, v, p = bufs[pick(i)]
+                ctx.slidedp_reduce_adamw_chunk(g, n, w, m, v, p, hp(wl, 1))
+        graph.replay()
+        torch.cuda.synchronize()
+        ev[0].record(st)
+        graph.replay()
+        ev[1].record(st)
+        torch.cuda.synchronize()
+        us = ev[0].elapsed_time(ev[1]) / reps * 1e3
+        res[name] = {"us_per_launch": us, "g_params_per_s": n / us / 1e3,
+                     "algorithmic_gbs": (26 + 2 * R) * n / us / 1e3}
+        del graph
+    res["note"] = ("320 launches replayed from one CUDA graph; the rotating case touches 16 x 31.5 MB = 504 MB "
+                   "(4 x L2) between reuses, the resident case is a cache number, not HBM")
+    out["tiny"] = res
+    del bufs
+
+    def pinned_state(n):
+        return [torch.empty(n, pin_memory=True) for _ in range(3)]
+
+    # ---- chunk-size sweep on the Qwen2.5-72B-shaped layer
+    wl = W.CONFIGS["qwen25_72b_layer_host"]
+    n, R = wl.numel, wl.R
+    grads = [W.rank_gradient(wl, r, step=wl.first_step, device=dev) for r in range(R)]
+    p = torch.zeros(n, dtype=torch.bfloat16, device=dev)
+    hw, hm, hv = pinned_state(n)
+    hw.copy_(W.master_weights(wl, device=dev)); hm.zero_(); hv.zero_()
+    dbuf = torch.empty(2 << 28, dtype=torch.float32, device=dev)
+    probes = {}
+    for mib in (16, 64, 256):
+        probes[str(mib)] = ctx.slidedp_link_probe(hm, hv, dbuf[:1 << 28], dbuf[1 << 28:],
+                                                  1 << 30, mib << 20, 3)
+    del dbuf
+    hm.zero_(); hv.zero_()
+    sweep, t = [], 1
+    for mib in wl.chunk_mib:
+        for nbuf in (2, 3):
+            runs = []
+            for i in range(4):
+                r_ = ctx.slidedp_stream_step(grads, n, hw, hm, hv, p, W.chunk_elems(mib), nbuf,
+                                             hp(wl, t))
+                t += 1
+                if i >= 1:
+                    runs.append(r_)
+            ms = statistics.mean(r_["ms_total"] for r_ in runs)
+            pr = probes[str(mib)]
+            bound = max(12.0 * n / (pr["h2d_bidir"] * 1e6), 12.0 * n / (pr["d2h_bidir"] * 1e6))
+            sweep.append({"chunk_mib": mib, "nbuf": nbuf, "ms_per_step": ms,
+                          "g_params_per_s": n / ms / 1e6,
+                          "link_gbs_each_way": 12.0 * n / (ms * 1e6), "frac_of_link": bound / ms,
+                          "lanes_ms": {k: statistics.mean(r_[k] for r_ in runs)
+                                       for k in ("ms_norm", "ms_h2d", "ms_kernel", "ms_d2h")}})
+    out["qwen25_72b_layer_host"] = {"params": n, "R": R, "link_probe_gbs": probes, "sweep": sweep}
+    del grads, p, hw, hm, hv
+    torch.cuda.empty_cache()
+
+    # ---- eight layers, R = 8: global norm over all layers, then every layer streamed
+    wl = W.CONFIGS["qwen3_14b_8layers_host"]
+    L, R, nl = wl.layers, wl.R, wl.layer_numel
+    grads = [[W.rank_gradient(wl, r, step=1, layer=l, device=dev) for r in range(R)]
+             for l in range(L)]
+    ps = [torch.zeros(nl, dtype=torch.bfloat16, device=dev) for _ in range(L)]
+    state = []
+    for l in range(L):
+        hw, hm, hv = pinned_state(nl)
+        hw.copy_(W.master_weights(wl, layer=l, device=dev)); hm.zero_(); hv.zero_()
+        state.append((hw, hm, hv))
+    ce = W.chunk_elems(64)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    step_ms, norm_ms = [], []
+    for t in range(1, wl.steps + 1):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        e0.record(st)
+        for l in range(L):
+            ctx.slidedp_grad_norm(grads[l], nl, 1.0 / R, l == 0)
+        ctx.slidedp_grad_norm_finish(wl.max_norm)
+        e1.record(st)
+        torch.cuda.synchronize()
+        for l in range(L):
+            ctx.slidedp_stream_step(grads[l], nl, *state[l], ps[l], ce, 3, hp(wl, t),
+                                    norm_ready=True, want_stats=False)
+        torch.cuda.synchronize()
+        step_ms.append((time.perf_counter() - t0) * 1e3)
+        norm_ms.append(e0.elapsed_time(e1))
+    ms = statistics.mean(step_ms[2:])
+    nm = statistics.mean(norm_ms[2:])
+    out["qwen3_14b_8layers_host"] = {
+        "params": wl.numel, "R": R, "layers": L, "steps": wl.steps, "chunk_mib": 64, "nbuf": 3,
+        "ms_per_step": ms, "g_params_per_s": wl.numel / ms / 1e6,
+        "link_gbs_each_way": 12.0 * wl.numel / (ms * 1e6),
+        "norm_pass_ms": nm, "norm_pass_gbs": 2.0 * R * wl.numel / (nm * 1e6),
+        "norm_pass_frac_of_hbm": 2.0 * R * wl.numel / (nm * 1e6) / peak,
+        "timing": "host wall clock per step bracketed by synchronize (the calls are synchronous)"}
+    ctx.slidedp_destroy()
+    print(json.dumps(out))
+    return 0
+
+
 def host_resident_report(ctx, sd, W, torch, dev):
     """Qwen3-14B-shaped layer with pinned host state, 64 MiB chunks, 3 slots, against the
     pinned-copy bandwidth measured in the same run."""
@@ -379,9 +518,12 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    ap.add_argument("--report", choices=["contract", "sweep"], default="contract")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.report == "sweep":
+        return run_sweep(args)
     return run_cuda(args)
 
 

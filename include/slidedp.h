@@ -75,8 +75,10 @@ typedef struct {
   double norm, clip_coef; /* the step's global norm and coefficient (0 and 1 if clipping off) */
   double ms_total;        /* first enqueue to last D2H complete                                */
   double ms_norm;         /* the norm pass when it ran inside the call                         */
-  double ms_h2d, ms_kernel, ms_d2h; /* summed busy time of each lane over all chunks          */
-  double gbs_h2d, gbs_d2h;          /* bytes moved / summed busy time of that lane            */
+  double ms_h2d;          /* copy-in lane: start of its first copy to end of its last copy    */
+  double ms_kernel;       /* update kernels: the first chunk's kernel time scaled to n_total   */
+  double ms_d2h;          /* copy-out lane: start of its first copy to end of its last copy   */
+  double gbs_h2d, gbs_d2h;/* bytes moved / that lane's span                                    */
   int64_t chunks;
   int32_t nonfinite;      /* 1 if the norm was inf or NaN                                      */
   int32_t reserved;

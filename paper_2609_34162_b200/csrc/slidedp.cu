@@ -20,8 +20,11 @@ namespace {
 constexpr double kWaitSeconds = 300.0;       // bound on every host-side wait
 constexpr int64_t kInitialPartials = 1 << 20;  // 8 MB: 2^20 tiles = 17 G parameters
 
+// Timing events of ONE kernel (the first chunk's). Per-chunk timing events, on the copy
+// streams or the compute stream, sit on the chunk's H2D -> kernel -> D2H chain and cost
+// several percent of link bandwidth at 16 MiB chunks, so a step records a fixed handful.
 struct ChunkEvents {
-  cudaEvent_t h2d_start, h2d_end, k_start, k_end, d2h_start, d2h_end;
+  cudaEvent_t k_start, k_end;
 };
 
 }  // namespace
@@ -47,6 +50,7 @@ struct slidedp_ctx {
   cudaEvent_t ev_updated[3] = {nullptr, nullptr, nullptr};
   cudaEvent_t ev_free[3] = {nullptr, nullptr, nullptr};
   cudaEvent_t ev_begin = nullptr, ev_norm_done = nullptr, ev_end = nullptr;
+  cudaEvent_t ev_in_first = nullptr, ev_in_last = nullptr, ev_out_first = nullptr, ev_out_last = nullptr;
   std::vector<ChunkEvents> timing;  // grown on demand, reused
 };
 
@@ -307,6 +311,10 @@ int slidedp_create(slidedp_ctx** out, int device, size_t gpu_budget_bytes) {
   step(cudaEventCreate(&ctx->ev_begin));
   step(cudaEventCreate(&ctx->ev_norm_done));
   step(cudaEventCreate(&ctx->ev_end));
+  step(cudaEventCreate(&ctx->ev_in_first));
+  step(cudaEventCreate(&ctx->ev_in_last));
+  step(cudaEventCreate(&ctx->ev_out_first));
+  step(cudaEventCreate(&ctx->ev_out_last));
   if (e == cudaSuccess) {
     const double init[4] = {0.0, 0.0, 1.0, 0.0};
     step(cudaMemcpy(ctx->scalars, init, sizeof init, cudaMemcpyHostToDevice));
@@ -333,10 +341,9 @@ int slidedp_destroy(slidedp_ctx* ctx) {
   for (cudaStream_t s : own) if (s) cudaStreamDestroy(s);
   auto kill = [](cudaEvent_t ev) { if (ev) cudaEventDestroy(ev); };
   kill(ctx->scalar_event); kill(ctx->ev_begin); kill(ctx->ev_norm_done); kill(ctx->ev_end);
+  kill(ctx->ev_in_first); kill(ctx->ev_in_last); kill(ctx->ev_out_first); kill(ctx->ev_out_last);
   for (int i = 0; i < 3; ++i) { kill(ctx->ev_loaded[i]); kill(ctx->ev_updated[i]); kill(ctx->ev_free[i]); }
-  for (ChunkEvents& c : ctx->timing) {
-    kill(c.h2d_start); kill(c.h2d_end); kill(c.k_start); kill(c.k_end); kill(c.d2h_start); kill(c.d2h_end);
-  }
+  for (ChunkEvents& c : ctx->timing) { kill(c.k_start); kill(c.k_end); }
   if (ctx->slots) cudaFree(ctx->slots);
   if (ctx->partials) cudaFree(ctx->partials);
   if (ctx->scalars) cudaFree(ctx->scalars);
@@ -441,11 +448,10 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
   }
   const int64_t nchunks = n_total == 0 ? 0 : (n_total + chunk_elems - 1) / chunk_elems;
   if (stats) {
-    while ((int64_t)ctx->timing.size() < nchunks) {
+    while (ctx->timing.empty() && nchunks > 0) {
       ChunkEvents c;
-      CU(cudaEventCreate(&c.h2d_start)); CU(cudaEventCreate(&c.h2d_end));
-      CU(cudaEventCreate(&c.k_start));   CU(cudaEventCreate(&c.k_end));
-      CU(cudaEventCreate(&c.d2h_start)); CU(cudaEventCreate(&c.d2h_end));
+      CU(cudaEventCreate(&c.k_start));
+      CU(cudaEventCreate(&c.k_end));
       ctx->timing.push_back(c);
     }
   }
@@ -472,14 +478,14 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
     float* sw = ctx->slots + (size_t)slot * 3 * cap;
     float* sm = sw + cap;
     float* sv = sm + cap;
-    ChunkEvents* te = stats ? &ctx->timing[c] : nullptr;
+    ChunkEvents* te = (stats && c == 0) ? &ctx->timing[0] : nullptr;
     // copy-in: the slot must have been drained by the copy-out of chunk c - nbuf
     if (c >= nbuf) CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_free[slot], 0));
-    if (te) CU(cudaEventRecord(te->h2d_start, ctx->s_in));
+    if (stats && c == 0) CU(cudaEventRecord(ctx->ev_in_first, ctx->s_in));
     CU(cudaMemcpyAsync(sw, host_master + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
     CU(cudaMemcpyAsync(sm, host_m + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
     CU(cudaMemcpyAsync(sv, host_v + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
-    if (te) CU(cudaEventRecord(te->h2d_end, ctx->s_in));
+    if (stats && c == nchunks - 1) CU(cudaEventRecord(ctx->ev_in_last, ctx->s_in));
     CU(cudaEventRecord(ctx->ev_loaded[slot], ctx->s_in));
     // update
     CU(cudaStreamWaitEvent(ctx->s_compute, ctx->ev_loaded[slot], 0));
@@ -492,11 +498,11 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
     CU(cudaEventRecord(ctx->ev_updated[slot], ctx->s_compute));
     // copy-out
     CU(cudaStreamWaitEvent(ctx->s_out, ctx->ev_updated[slot], 0));
-    if (te) CU(cudaEventRecord(te->d2h_start, ctx->s_out));
+    if (stats && c == 0) CU(cudaEventRecord(ctx->ev_out_first, ctx->s_out));
     CU(cudaMemcpyAsync(host_master + off, sw, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
     CU(cudaMemcpyAsync(host_m + off, sm, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
     CU(cudaMemcpyAsync(host_v + off, sv, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
-    if (te) CU(cudaEventRecord(te->d2h_end, ctx->s_out));
+    if (stats && c == nchunks - 1) CU(cudaEventRecord(ctx->ev_out_last, ctx->s_out));
     CU(cudaEventRecord(ctx->ev_free[slot], ctx->s_out));
   }
   // the step ends when the compute stream (norm, even with no chunks) and the last
@@ -519,11 +525,15 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
     CU(cudaEventElapsedTime(&ms, ctx->ev_begin, ctx->ev_norm_done));
     stats->ms_norm = (clip && !norm_ready) ? ms : 0.0;
     stats->chunks = nchunks;
-    for (int64_t c = 0; c < nchunks; ++c) {
-      const ChunkEvents& te = ctx->timing[c];
-      CU(cudaEventElapsedTime(&ms, te.h2d_start, te.h2d_end)); stats->ms_h2d += ms;
-      CU(cudaEventElapsedTime(&ms, te.k_start, te.k_end));     stats->ms_kernel += ms;
-      CU(cudaEventElapsedTime(&ms, te.d2h_start, te.d2h_end)); stats->ms_d2h += ms;
+    if (nchunks > 0) {
+      const ChunkEvents& te = ctx->timing[0];
+      const int64_t first_len = n_total < chunk_elems ? n_total : chunk_elems;
+      CU(cudaEventElapsedTime(&ms, te.k_start, te.k_end));
+      stats->ms_kernel = (double)ms * ((double)n_total / (double)first_len);
+      CU(cudaEventElapsedTime(&ms, ctx->ev_in_first, ctx->ev_in_last));
+      stats->ms_h2d = ms;
+      CU(cudaEventElapsedTime(&ms, ctx->ev_out_first, ctx->ev_out_last));
+      stats->ms_d2h = ms;
     }
     const double link_bytes = 12.0 * (double)n_total;
     if (stats->ms_h2d > 0) stats->gbs_h2d = link_bytes / (stats->ms_h2d * 1e6);

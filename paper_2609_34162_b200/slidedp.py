@@ -215,3 +215,4 @@ class Context:
 
 def slidedp_create(device: int = 0, gpu_budget_bytes: int = 0) -> Context:
     return Context(device, gpu_budget_bytes)
+

@@ -56,7 +56,8 @@ typedef enum {
   SLIDEDP_ERR_NOT_PINNED = -4,  /* a host state pointer of slidedp_stream_step is not page-locked      */
   SLIDEDP_ERR_CUDA = -5,        /* a CUDA runtime call failed; see slidedp_last_cuda_error()            */
   SLIDEDP_ERR_TIMEOUT = -6,     /* a bounded wait for queued work expired                               */
-  SLIDEDP_ERR_NO_NORM = -7      /* clipping requested but no finished norm is held by the context      */
+  SLIDEDP_ERR_NO_NORM = -7,     /* clipping requested but no finished norm is held by the context      */
+  SLIDEDP_ERR_TOO_LARGE = -8    /* n exceeds the fixed capacity of slidedp_grad_norm_noalloc            */
 } slidedp_status;
 
 typedef struct slidedp_ctx slidedp_ctx;
@@ -171,6 +172,37 @@ SLIDEDP_API int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_b
  */
 SLIDEDP_API int slidedp_link_probe(slidedp_ctx* ctx, void* host_a, void* host_b, void* dev_a, void* dev_b,
                        size_t bytes, size_t copy_bytes, int reps, double out4[4]);
+
+/* ---- global norm for callers that cannot allocate ---------------------------------------
+ *
+ * (No counterpart in the paper: this entry point exists for deployment reasons only.)
+ * Some callers may not allocate device memory at the moment they need the norm, or ever: code
+ * running inside a memory-pool or allocator callback, a host process whose memory budget is
+ * fixed and fully handed out at start-up, or a plug-in that is only given pointers. Such
+ * callers cannot use slidedp_create (it allocates the workspace of slidedp_grad_norm).
+ * slidedp_grad_norm_noalloc computes the same quantity as slidedp_grad_norm followed by
+ * slidedp_grad_norm_finish for ONE chunk, with the same kernels, tiling and summation tree
+ * (so the same bits), but keeps its tile sums in a fixed array compiled into the library's
+ * device image instead of allocated memory. It takes no context and calls no cudaMalloc,
+ * cudaFree or any allocating routine.
+ *
+ * grads_bf16: host array of R device pointers (16-byte aligned) to n BF16 values each, on the
+ * CURRENT device. out4: device pointer (16-byte aligned) to four doubles that receive sumsq,
+ * norm, coef = max_norm > 0 ? min(1, max_norm/(norm + 1e-6)) : 1, and 1.0 if the norm is not
+ * finite (else 0.0). Asynchronous on cuda_stream.
+ *
+ * Limits and sharing: n <= SLIDEDP_NOALLOC_MAX_ELEMS (2^30); more gives
+ * SLIDEDP_ERR_TOO_LARGE and nothing is launched. The array (512 KiB) is held by every GPU
+ * that loads the library until the process exits. All calls on a device share it: two calls
+ * whose kernels may overlap on the GPU (different streams without ordering) race on it; calls
+ * ordered on one stream are safe. It keeps the previous call's tile sums, and nothing has to
+ * start at zero: each call overwrites the tiles it then reads and reads no others.
+ * The first call on each device looks up the array's device address (a one-time set-up with
+ * that device current); make that first call before starting any stream capture.
+ */
+#define SLIDEDP_NOALLOC_MAX_ELEMS ((int64_t)1 << 30)
+SLIDEDP_API int slidedp_grad_norm_noalloc(const void* const* grads_bf16, int R, int64_t n, double inv_R,
+                              double max_norm, double* out4, void* cuda_stream);
 
 /* Number of kernels this library has launched on the context since creation. */
 SLIDEDP_API int64_t slidedp_kernel_launches(const slidedp_ctx* ctx);

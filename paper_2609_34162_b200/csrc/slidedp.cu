@@ -269,6 +269,7 @@ const char* slidedp_strerror(int status) {
     case SLIDEDP_ERR_CUDA: return "a CUDA call failed";
     case SLIDEDP_ERR_TIMEOUT: return "a bounded wait expired";
     case SLIDEDP_ERR_NO_NORM: return "clipping requested before any norm was finished";
+    case SLIDEDP_ERR_TOO_LARGE: return "n exceeds the fixed capacity of the no-allocation entry point";
     default: return "unknown status";
   }
 }
@@ -609,6 +610,63 @@ int slidedp_link_probe(slidedp_ctx* ctx, void* host_a, void* host_b, void* dev_a
   }
   cudaEventDestroy(a0); cudaEventDestroy(a1); cudaEventDestroy(b0); cudaEventDestroy(b1);
   return rc;
+}
+
+// ---- norm without allocation ---------------------------------------------------------------
+//
+// Scratch for callers that cannot allocate: the per-tile sums live in an array that is part
+// of the library's device image. In HOST code the name `noalloc_tile_sums` is only a handle
+// for the symbol, not a device address; the address each device gave it is looked up once
+// per device with cudaGetSymbolAddress (with that device current) and cached here.
+constexpr int64_t kNoallocMaxTiles = SLIDEDP_NOALLOC_MAX_ELEMS / kNormTile;   // 65536
+static __device__ __align__(256) double noalloc_tile_sums[kNoallocMaxTiles];
+
+constexpr int kNoallocMaxDevices = 64;
+static double* noalloc_scratch_addr[kNoallocMaxDevices];   // zero-initialised: not looked up yet
+
+int slidedp_grad_norm_noalloc(const void* const* grads_bf16, int R, int64_t n, double inv_R,
+                              double max_norm, double* out4, void* cuda_stream) {
+  if (n < 0 || !out4 || inv_R != inv_R || max_norm != max_norm) return SLIDEDP_ERR_INVALID_ARG;
+  GradPtrs gp;
+  int rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  if (!aligned16(out4)) return SLIDEDP_ERR_MISALIGNED;
+  if (n > SLIDEDP_NOALLOC_MAX_ELEMS) return SLIDEDP_ERR_TOO_LARGE;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return SLIDEDP_ERR_CUDA; }
+  if (dev < 0 || dev >= kNoallocMaxDevices) return SLIDEDP_ERR_INVALID_ARG;
+  double* scratch = noalloc_scratch_addr[dev];
+  if (!scratch) {
+    // one-time set-up for this device (current right now): resolve the symbol's address
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, noalloc_tile_sums) != cudaSuccess || !p) {
+      (void)cudaGetLastError();
+      return SLIDEDP_ERR_CUDA;
+    }
+    scratch = static_cast<double*>(p);
+    noalloc_scratch_addr[dev] = scratch;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
+  if (ntiles > 0) {
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int64_t max_blocks = (int64_t)sms * 8;
+    const unsigned blocks = (unsigned)(ntiles < max_blocks ? ntiles : max_blocks);
+    const float inv = (float)inv_R;
+    switch (R) {
+      case 1: grad_sumsq_tiles_kernel<1><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, scratch); break;
+      case 2: grad_sumsq_tiles_kernel<2><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, scratch); break;
+      case 4: grad_sumsq_tiles_kernel<4><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, scratch); break;
+      case 8: grad_sumsq_tiles_kernel<8><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, scratch); break;
+      default: grad_sumsq_tiles_kernel<0><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, scratch); break;
+    }
+    if (cudaGetLastError() != cudaSuccess) return SLIDEDP_ERR_CUDA;
+  }
+  // reads tiles [0, ntiles) only: whatever an earlier call left beyond them is never seen
+  grad_norm_finish_kernel<<<1, kFinishThreads, 0, st>>>(scratch, ntiles, max_norm, out4);
+  if (cudaGetLastError() != cudaSuccess) return SLIDEDP_ERR_CUDA;
+  return SLIDEDP_OK;
 }
 
 }  // extern "C"

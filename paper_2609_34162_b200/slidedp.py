@@ -26,6 +26,8 @@ _lib = ctypes.CDLL(LIB_PATH)
 MAX_RANKS = 16
 OK, ERR_INVALID_ARG, ERR_MISALIGNED, ERR_BUDGET, ERR_NOT_PINNED, ERR_CUDA, ERR_TIMEOUT, ERR_NO_NORM = (
     0, -1, -2, -3, -4, -5, -6, -7)
+ERR_TOO_LARGE = -8
+NOALLOC_MAX_ELEMS = 1 << 30
 
 
 class _HParams(ctypes.Structure):
@@ -87,6 +89,9 @@ _lib.slidedp_stream_step.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp
 _lib.slidedp_link_probe.restype = ctypes.c_int
 _lib.slidedp_link_probe.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, ctypes.c_size_t,
                                     ctypes.c_int, ctypes.POINTER(ctypes.c_double)]
+_lib.slidedp_grad_norm_noalloc.restype = ctypes.c_int
+_lib.slidedp_grad_norm_noalloc.argtypes = [_pp, ctypes.c_int, ctypes.c_int64, ctypes.c_double,
+                                           ctypes.c_double, _vp, _vp]
 _lib.slidedp_kernel_launches.restype = ctypes.c_int64
 _lib.slidedp_kernel_launches.argtypes = [_vp]
 
@@ -216,3 +221,18 @@ class Context:
 def slidedp_create(device: int = 0, gpu_budget_bytes: int = 0) -> Context:
     return Context(device, gpu_budget_bytes)
 
+
+def slidedp_grad_norm_noalloc(grads, n: int, inv_R: float, max_norm: float, out4, stream=None) -> None:
+    """Global norm of one chunk for callers that must not allocate device memory (allocator
+    callbacks, processes with a fully committed memory budget, plug-ins that only receive
+    pointers): same result as ``slidedp_grad_norm`` + ``slidedp_grad_norm_finish``, but the
+    tile sums live in a fixed 512 KiB array inside the library instead of a context.
+
+    ``out4`` is a caller-owned device tensor of four float64 (sumsq, norm, coef, non-finite
+    flag). ``n`` may not exceed ``NOALLOC_MAX_ELEMS``. Calls share the array, so only issue
+    them ordered on one stream; make the first call on a device outside any stream capture.
+    """
+    rc = _lib.slidedp_grad_norm_noalloc(_grad_array(grads), len(grads), n, inv_R, max_norm,
+                                        _ptr(out4), _stream(stream))
+    if rc != OK:
+        raise SlideDPError(rc)

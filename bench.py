@@ -144,6 +144,28 @@ def run_reference(args):
     return 0
 
 
+# ------------------------------------------------------------------ multi-rank plumbing
+def layer_of_rank(rank: int) -> int:
+    """Every rank owns a different layer (an independent partition of the model)."""
+    return rank
+
+
+def max_over_ranks(x: float, world: int, device="cuda") -> float:
+    """The slowest rank's time: multi-GPU numbers are device times, max over ranks."""
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world: int, params_per_rank: int, steps: int, total_ms: float) -> float:
+    """Whole-job G-params/s: the parameters all ranks updated over the slowest rank's time."""
+    return world * params_per_rank * steps / (total_ms * 1e-3) / 1e9
+
+
 # --------------------------------------------------------------------------------- CUDA arm
 def run_cuda(args):
     import numpy as np
@@ -168,16 +190,9 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
     wl = W.CONFIGS[WORKLOAD]
     n, R = wl.numel, wl.R
-    layer = rank                                   # every rank owns a different layer
+    layer = layer_of_rank(rank)
     ctx = sd.slidedp_create(local, 0)
     stream = torch.cuda.current_stream()
     dev = torch.device("cuda", local)
@@ -232,14 +247,14 @@ def run_cuda(args):
     stop.record(stream)
     barrier()
     launches = ctx.slidedp_kernel_launches() - launches0
-    total_ms = max_over_ranks(start.elapsed_time(stop))
+    total_ms = max_over_ranks(start.elapsed_time(stop), world)
     norm_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in events)
     upd_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in events)
     upd_best = min(e[1].elapsed_time(e[2]) for e in events)
     t_next += args.steps
 
     ms_per_step = total_ms / args.steps
-    value = world * n / (ms_per_step * 1e-3) / 1e9
+    value = job_value(world, n, args.steps, total_ms)
     peak, peak_kind = measured_peak_hbm()
     upd_bytes = (26 + 2 * R) * n
     achieved = upd_bytes / (upd_ms * 1e-3) / 1e9
@@ -273,8 +288,8 @@ def run_cuda(args):
     wall = time.perf_counter() - wall0
     barrier()
     t_next += e2e_steps
-    e2e_ms = max_over_ranks(e2e_ms)
-    e2e = {"value": world * n * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+    e2e_ms = max_over_ranks(e2e_ms, world)
+    e2e = {"value": job_value(world, n, e2e_steps, e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": 12 * n, "d2h_bytes_per_step": 12 * n + 32,
            "ms_per_step": e2e_ms / e2e_steps, "wall_ms_per_step": wall / e2e_steps * 1e3,
            "steps": e2e_steps, "chunk_mib": 64, "nbuf": 3,

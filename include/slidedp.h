@@ -156,6 +156,9 @@ SLIDEDP_API int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* 
  * already held by the context (a step that spans several calls: run slidedp_grad_norm over
  * every layer and slidedp_grad_norm_finish first). Synchronous: returns after the last
  * copy-out completed (bounded wait, SLIDEDP_ERR_TIMEOUT). stats is nullable.
+ * The call runs on the context's own non-blocking streams and does not order itself after
+ * any stream of the caller: whatever produced the gradients, and with norm_ready the
+ * slidedp_grad_norm_finish, must have completed (synchronise that stream first).
  * Link traffic is 12 bytes per parameter in each direction.
  */
 SLIDEDP_API int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n_total,

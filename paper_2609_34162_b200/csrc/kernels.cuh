@@ -168,7 +168,7 @@ reduce_adamw_kernel(GradPtrs gp, int R_rt, int64_t n, float* __restrict__ master
 // adds its 8 * kNormIters squares in index order, the warp folds by an xor butterfly
 // (16, 8, 4, 2, 1), and thread 0 adds the 8 warp sums in warp order: the tree is fixed, so
 // a tile's partial does not depend on which block computes it or on the grid size.
-template <int R_T>
+template <int R_T, int UNROLL = 4>
 __global__ void __launch_bounds__(kNormThreads)
 grad_sumsq_tiles_kernel(GradPtrs gp, int R_rt, int64_t n, float inv_R,
                         double* __restrict__ partials) {
@@ -178,7 +178,7 @@ grad_sumsq_tiles_kernel(GradPtrs gp, int R_rt, int64_t n, float inv_R,
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     const int64_t tbase = tile * kNormTile + (int64_t)threadIdx.x * kNormVec;
     double acc = 0.0;
-#pragma unroll 4
+#pragma unroll UNROLL
     for (int it = 0; it < kNormIters; ++it) {
       const int64_t e = tbase + (int64_t)it * (kNormThreads * kNormVec);
       float s[kNormVec];

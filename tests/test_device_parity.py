@@ -251,3 +251,46 @@ def test_argument_errors_are_reported_not_faulted(ctx, sd):
         fresh.slidedp_destroy()
     torch.cuda.synchronize()
     assert torch.all(w == 0)
+
+
+def test_indices_beyond_2_to_31(ctx, sd):
+    """A chunk of 2^31 + 4099 parameters (34 GB on the device): 64-bit indexing in both kernels.
+    The update is elementwise, so the oracle checks slices (head, around 2^31, ragged tail) with
+    the global coefficient; the norm is checked over the whole range."""
+    n, R = (1 << 31) + 4099, 1
+    free, _ = torch.cuda.mem_get_info()
+    if free < 45 << 30:
+        pytest.skip("needs 45 GB of free device memory")
+    gen = torch.Generator(device="cuda").manual_seed(2031)
+    g = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    w = torch.empty(n, device="cuda")
+    seg = 1 << 27
+    for lo in range(0, n, seg):
+        k = min(seg, n - lo)
+        g[lo:lo + k] = (torch.randn(k, generator=gen, device="cuda") * 1e-3).to(torch.bfloat16)
+        w[lo:lo + k] = torch.randn(k, generator=gen, device="cuda") * 0.02
+    m = w * 0.01
+    v = w * w * 1e-3
+    p = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    slices = [(0, 1 << 20), ((1 << 31) - (1 << 19), (1 << 31) + (1 << 19)), (n - (1 << 20), n)]
+    before = [[parity.f32(t[a:b]).copy() for t in (w, m, v)] for a, b in slices]
+    kw = dict(ADAM, inv_R=1.0, max_norm=1.0, step=11)
+    ctx.slidedp_grad_norm([g], n, 1.0, True)
+    norm_g, coef_g = ctx.slidedp_grad_norm_finish(1.0, fetch=True)
+    ctx.slidedp_reduce_adamw_chunk([g], n, w, m, v, p, sd.HParams(**kw))
+    torch.cuda.synchronize()
+    hg = parity.u16(g)
+    coef_o, norm_o = oracle.clip_coef(oracle.grad_sumsq([hg], 1.0, NTHREADS), 1.0)
+    parity.assert_norm_close(norm_g, norm_o)
+    assert coef_o < 1.0 and abs(coef_g - coef_o) <= 1e-6 * coef_o
+    for (a, b), (ow, om, ov) in zip(slices, before):
+        op = np.zeros(b - a, np.uint16)
+        oracle.reduce_adamw_chunk([hg[a:b].copy()], ow, om, ov, op, oracle.HParams(**kw),
+                                  clip=coef_o, nthreads=NTHREADS)
+        tag = f"[{a}:{b}]"
+        parity.assert_fp32_close(tag + "/master", parity.f32(w[a:b]), ow)
+        parity.assert_fp32_close(tag + "/m", parity.f32(m[a:b]), om)
+        parity.assert_fp32_close(tag + "/v", parity.f32(v[a:b]), ov)
+        parity.assert_bf16_close(tag + "/param_bf16", parity.u16(p[a:b]), op)
+    # nothing outside the chunk was touched and every element inside was written
+    assert int((p == 0).sum()) < n // 1000

@@ -415,11 +415,17 @@ def run_sweep(args):
             ms = statistics.mean(r_["ms_total"] for r_ in runs)
             pr = probes[str(mib)]
             bound = max(12.0 * n / (pr["h2d_bidir"] * 1e6), 12.0 * n / (pr["d2h_bidir"] * 1e6))
+            lanes = {k: statistics.mean(r_[k] for r_ in runs)
+                     for k in ("ms_norm", "ms_h2d", "ms_kernel", "ms_d2h")}
+            # the paper's dependency model fed with rates measured in this run
+            lo_ms, pred_ms = sd.slidedp_model_stream_step(
+                n, R, W.chunk_elems(mib), nbuf, pr["h2d_bidir"], pr["d2h_bidir"],
+                n / (lanes["ms_kernel"] * 1e6), 2.0 * R * n / (lanes["ms_norm"] * 1e6), 3.0)
             sweep.append({"chunk_mib": mib, "nbuf": nbuf, "ms_per_step": ms,
+                          "model_lower_bound_ms": lo_ms, "model_predicted_ms": pred_ms,
                           "g_params_per_s": n / ms / 1e6,
                           "link_gbs_each_way": 12.0 * n / (ms * 1e6), "frac_of_link": bound / ms,
-                          "lanes_ms": {k: statistics.mean(r_[k] for r_ in runs)
-                                       for k in ("ms_norm", "ms_h2d", "ms_kernel", "ms_d2h")}})
+                          "lanes_ms": lanes})
     out["qwen25_72b_layer_host"] = {"params": n, "R": R, "link_probe_gbs": probes, "sweep": sweep}
     del grads, p, hw, hm, hv
     torch.cuda.empty_cache()
@@ -494,7 +500,14 @@ def host_resident_report(ctx, sd, W, torch, dev):
     ms = statistics.mean(r["ms_total"] for r in runs)
     link_bytes = 12.0 * n
     bound_ms = max(link_bytes / (probe["h2d_bidir"] * 1e6), link_bytes / (probe["d2h_bidir"] * 1e6))
-    return {"workload": HOST_WORKLOAD, "params": n, "R": R, "chunk_mib": 64, "nbuf": 3,
+    # parameter delivery (the step before the path): BF16 copy of the pinned FP32 master
+    dl = [ctx.slidedp_deliver_params(hw, n, p, ce, 3) for _ in range(4)][1:]
+    dl_ms = statistics.mean(r["ms_total"] for r in dl)
+    delivery = {"ms": dl_ms, "g_params_per_s": n / dl_ms / 1e6, "h2d_bytes": 4 * n,
+                "roofline": {"bound": "host-link", "unit": "GB/s", "achieved": 4.0 * n / (dl_ms * 1e6),
+                             "peak": probe["h2d"], "frac": 4.0 * n / (dl_ms * 1e6) / probe["h2d"],
+                             "peak_source": "pinned-copy probe in this run, H2D alone"}}
+    return {"workload": HOST_WORKLOAD, "delivery": delivery, "params": n, "R": R, "chunk_mib": 64, "nbuf": 3,
             "value": n / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
             "link_probe_gbs": probe,
             "link_gbs_effective_each_way": link_bytes / (ms * 1e6),

@@ -166,6 +166,49 @@ SLIDEDP_API int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_b
                         void* param_bf16_out, int64_t chunk_elems, int nbuf, int norm_ready,
                         const slidedp_hparams* hp, slidedp_stats* stats);
 
+/* ---- parameter delivery: BF16 copy of a host-resident FP32 master -------------------------
+ *
+ * The step BEFORE the update path (paper Sec. 3.3 "Overlap within a layer": on parameter
+ * delivery chunk k+1 is cast to BF16 while DMA transfers chunk k; Sec. 3.2 "Parameter
+ * dispatch"). The paper casts on the CPU and moves BF16 (2 bytes per parameter); here the
+ * pinned FP32 master is copied H2D chunk by chunk (4 bytes per parameter) into the context's
+ * slots and cast on the GPU, copy of chunk k+1 overlapping the cast of chunk k, so no host core
+ * and no host DRAM bandwidth beyond the DMA read is spent:
+ *   param_bf16_out[i] = bf16_round_to_nearest_even(host_master[i])        for i in [0, n_total)
+ * host_master: PINNED, n_total floats, read-only. param_bf16_out: device, n_total BF16.
+ * chunk_elems: multiple of 8; nbuf 2 or 3; slots take nbuf * chunk_elems * 4 bytes under the
+ * context's budget (SLIDEDP_ERR_BUDGET). Synchronous (bounded wait); runs on the context's own
+ * streams like slidedp_stream_step. stats (nullable): ms_total, ms_h2d / gbs_h2d (copy lane
+ * span and 4 n_total bytes over it), chunks; the other fields are zero.
+ */
+SLIDEDP_API int slidedp_deliver_params(slidedp_ctx* ctx, const float* host_master, int64_t n_total,
+                           void* param_bf16_out, int64_t chunk_elems, int nbuf,
+                           slidedp_stats* stats);
+
+/* ---- step-time model of the host-resident step (host arithmetic only, no GPU work) --------
+ *
+ * The paper's dependency model (Sec. 3.4 "Modeling Shared-Host Scaling") applied to
+ * slidedp_stream_step. Resource demand gives the lower bound  T >= max_j W_j / beta_j  over the
+ * copy-in lane, the copy-out lane and the compute lane; execution dependencies give each
+ * operation's completion  f(v) = d_v + max({a_v} U {f(u) : u in P(v)})  with
+ *   copy-in  of chunk k after copy-in  of k-1 (stream order) and copy-out of k-nbuf (buffer),
+ *   kernel   of chunk k after copy-in  of k   (data) and kernel of k-1 (stream; the norm pass
+ *            precedes kernel 0),
+ *   copy-out of chunk k after kernel   of k   (data) and copy-out of k-1 (stream).
+ * d_v = bytes / rate (+ per_copy_us for each of a chunk's three copies); all release times
+ * a_v are 0. Rates are what slidedp_link_probe and the kernel benchmarks measured.
+ * Writes the bound and the predicted completion of the last copy-out, in ms.
+ */
+typedef struct {
+  double h2d_gbs, d2h_gbs;      /* link rates while both directions are busy (GB/s)         */
+  double update_gparams_s;      /* fused update kernel rate on device slots (G-params/s)    */
+  double norm_gbs;              /* norm pass rate over the gradients (GB/s); 0: no norm pass */
+  double per_copy_us;           /* fixed cost of one cudaMemcpyAsync on its lane (us)        */
+} slidedp_rates;
+SLIDEDP_API int slidedp_model_stream_step(int64_t n_total, int R, int64_t chunk_elems, int nbuf,
+                              const slidedp_rates* rates, double* lower_bound_ms,
+                              double* predicted_ms);
+
 /* ---- host-link probe: the roofline of the host-resident mode ---------------------------
  *
  * Copies `bytes` between a pinned host buffer and a device buffer in pieces of copy_bytes,

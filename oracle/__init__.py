@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
                                   ctypes.c_int64, ctypes.POINTER(_HParams),
                                   ctypes.POINTER(ctypes.c_double),
                                   ctypes.POINTER(ctypes.c_double), ctypes.c_int]
+        L.oracle_cast_master_to_bf16.restype = None
+        L.oracle_cast_master_to_bf16.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
         L.oracle_max_threads.restype = ctypes.c_int
         L.oracle_max_threads.argtypes = []
         _lib = L
@@ -150,6 +152,13 @@ def clip_coef(sumsq: float, max_norm: float):
     norm = ctypes.c_double()
     c = lib().oracle_clip_coef(sumsq, max_norm, ctypes.byref(norm))
     return float(c), float(norm.value)
+
+
+def cast_master_to_bf16(master: np.ndarray) -> np.ndarray:
+    _check(master, np.float32)
+    out = np.empty(master.size, np.uint16)
+    lib().oracle_cast_master_to_bf16(master.ctypes.data, master.size, out.ctypes.data)
+    return out
 
 
 def reduce_adamw_chunk(grads, master, m, v, param_bf16, hp: HParams, clip: float = 1.0,

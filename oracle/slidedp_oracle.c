@@ -158,6 +158,10 @@ int oracle_step(const uint16_t* const* grads, int R, int64_t n_total,
   return 0;
 }
 
+void oracle_cast_master_to_bf16(const float* master, int64_t n, uint16_t* param_bf16) {
+  for (int64_t i = 0; i < n; ++i) param_bf16[i] = oracle_f32_to_bf16(master[i]);
+}
+
 int oracle_max_threads(void) {
 #ifdef _OPENMP
   return omp_get_max_threads();

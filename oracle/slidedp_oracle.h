@@ -87,6 +87,10 @@ int oracle_step(const uint16_t* const* grads, int R, int64_t n_total,
                 int64_t chunk_elems, const oracle_hparams* hp,
                 double* norm_out, double* coef_out, int nthreads);
 
+/* Parameter delivery (paper Sec. 3.3 "Overlap within a layer": the FP32 master is cast to BF16
+ * for the next delivery): p[i] = round-to-nearest-even BF16 of master[i]. */
+void oracle_cast_master_to_bf16(const float* master, int64_t n, uint16_t* param_bf16);
+
 /* Threads an nthreads > 1 call would really use (1 when built without OpenMP). */
 int oracle_max_threads(void);
 

@@ -168,7 +168,9 @@ reduce_adamw_kernel(GradPtrs gp, int R_rt, int64_t n, float* __restrict__ master
 // adds its 8 * kNormIters squares in index order, the warp folds by an xor butterfly
 // (16, 8, 4, 2, 1), and thread 0 adds the 8 warp sums in warp order: the tree is fixed, so
 // a tile's partial does not depend on which block computes it or on the grid size.
-template <int R_T, int UNROLL = 4>
+// Launched with one block per tile; the loads of UNROLL iterations are in flight together
+// (measured best: 2 at R = 4, 1 at R = 8, where more unrolling costs occupancy).
+template <int R_T, int UNROLL = (R_T == 0 || R_T >= 8) ? 1 : (R_T >= 4 ? 2 : 4)>
 __global__ void __launch_bounds__(kNormThreads)
 grad_sumsq_tiles_kernel(GradPtrs gp, int R_rt, int64_t n, float inv_R,
                         double* __restrict__ partials) {
@@ -261,6 +263,30 @@ grad_norm_finish_kernel(const double* __restrict__ partials, int64_t count, doub
     scalars[1] = norm;
     scalars[2] = c;
     scalars[3] = (norm - norm == 0.0) ? 0.0 : 1.0;
+  }
+}
+
+// ---- parameter delivery: FP32 master -> BF16 copy --------------------------------------
+//
+// Eight elements per thread: two 16-byte loads, one 16-byte store, round to nearest even.
+// HBM traffic is 6 bytes per parameter, but the kernel always runs behind an H2D copy of the
+// same chunk (4 bytes per parameter over the host link), which is the bound.
+constexpr int kCastThreads = 256;
+__global__ void __launch_bounds__(kCastThreads)
+cast_master_to_bf16_kernel(const float* __restrict__ master, int64_t n,
+                           uint16_t* __restrict__ param_out) {
+  const int64_t base = ((int64_t)blockIdx.x * kCastThreads + threadIdx.x) * 8;
+  if (base >= n) return;
+  if (base + 8 <= n) {
+    const uint4 a = ld_stream(master + base), b = ld_stream(master + base + 4);
+    uint4 o;
+    o.x = f32_to_bf16_bits(__uint_as_float(a.x)) | (f32_to_bf16_bits(__uint_as_float(a.y)) << 16);
+    o.y = f32_to_bf16_bits(__uint_as_float(a.z)) | (f32_to_bf16_bits(__uint_as_float(a.w)) << 16);
+    o.z = f32_to_bf16_bits(__uint_as_float(b.x)) | (f32_to_bf16_bits(__uint_as_float(b.y)) << 16);
+    o.w = f32_to_bf16_bits(__uint_as_float(b.z)) | (f32_to_bf16_bits(__uint_as_float(b.w)) << 16);
+    st_stream(param_out + base, o);
+  } else {
+    for (int64_t i = base; i < n; ++i) param_out[i] = (uint16_t)f32_to_bf16_bits(master[i]);
   }
 }
 

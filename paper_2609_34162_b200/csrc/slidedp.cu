@@ -205,10 +205,8 @@ int norm_chunk(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, double in
   const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
   int rc = ensure_partials(ctx, ctx->partials_used + ntiles, st);
   if (rc != SLIDEDP_OK) return rc;
-  int sms = 148;
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
-  const int64_t max_blocks = (int64_t)sms * 8;
-  const unsigned blocks = (unsigned)(ntiles < max_blocks ? ntiles : max_blocks);
+  // one block per tile: the hardware scheduler balances them, a tail of one tile at most
+  const unsigned blocks = (unsigned)ntiles;
   double* dst = ctx->partials + ctx->partials_used;
   const float inv = (float)inv_R;
   switch (R) {
@@ -239,6 +237,17 @@ int fetch_scalars(slidedp_ctx* ctx, cudaStream_t st) {
                      cudaMemcpyDeviceToHost, st));
   CU(cudaEventRecord(ctx->scalar_event, st));
   return bounded_event_wait(ctx, ctx->scalar_event, kWaitSeconds);
+}
+
+// Grows the slot allocation to `need` bytes if the budget allows (checked before any work).
+int ensure_slots(slidedp_ctx* ctx, size_t need) {
+  if (ctx->budget && need > ctx->budget) return SLIDEDP_ERR_BUDGET;
+  if (need > ctx->slot_bytes) {
+    if (ctx->slots) { CU(cudaFree(ctx->slots)); ctx->slots = nullptr; ctx->slot_bytes = 0; }
+    CU(cudaMalloc(&ctx->slots, need));
+    ctx->slot_bytes = need;
+  }
+  return SLIDEDP_OK;
 }
 
 int is_pinned(slidedp_ctx* ctx, const void* p, bool* pinned) {
@@ -441,12 +450,8 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
   // slots: nbuf x {master, m, v} x cap floats
   const int64_t cap = chunk_elems < n_total ? chunk_elems : ((n_total + 7) / 8) * 8;
   const size_t need = (size_t)nbuf * 3 * (size_t)cap * sizeof(float);
-  if (ctx->budget && need > ctx->budget) return SLIDEDP_ERR_BUDGET;
-  if (need > ctx->slot_bytes) {
-    if (ctx->slots) { CU(cudaFree(ctx->slots)); ctx->slots = nullptr; ctx->slot_bytes = 0; }
-    CU(cudaMalloc(&ctx->slots, need));
-    ctx->slot_bytes = need;
-  }
+  rc = ensure_slots(ctx, need);
+  if (rc != SLIDEDP_OK) return rc;
   const int64_t nchunks = n_total == 0 ? 0 : (n_total + chunk_elems - 1) / chunk_elems;
   if (stats) {
     while (ctx->timing.empty() && nchunks > 0) {
@@ -545,6 +550,113 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
       stats->nonfinite = ctx->host_scalars[3] != 0.0;
     }
   }
+  return SLIDEDP_OK;
+}
+
+int slidedp_deliver_params(slidedp_ctx* ctx, const float* host_master, int64_t n_total,
+                           void* param_bf16_out, int64_t chunk_elems, int nbuf,
+                           slidedp_stats* stats) {
+  if (!ctx || n_total < 0) return SLIDEDP_ERR_INVALID_ARG;
+  if (nbuf < 2 || nbuf > 3 || chunk_elems <= 0 || (chunk_elems % 8) != 0)
+    return SLIDEDP_ERR_INVALID_ARG;
+  if (n_total > 0 && (!host_master || !param_bf16_out)) return SLIDEDP_ERR_INVALID_ARG;
+  if (!aligned16(host_master) || !aligned16(param_bf16_out)) return SLIDEDP_ERR_MISALIGNED;
+  if (stats) {
+    memset(stats, 0, sizeof *stats);
+    stats->clip_coef = 1.0;
+  }
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  int rc = SLIDEDP_OK;
+  if (n_total > 0) {
+    bool pinned = false;
+    rc = is_pinned(ctx, host_master, &pinned);
+    if (rc != SLIDEDP_OK) return rc;
+    if (!pinned) return SLIDEDP_ERR_NOT_PINNED;
+  }
+  const int64_t cap = chunk_elems < n_total ? chunk_elems : ((n_total + 7) / 8) * 8;
+  rc = ensure_slots(ctx, (size_t)nbuf * (size_t)cap * sizeof(float));
+  if (rc != SLIDEDP_OK) return rc;
+  const int64_t nchunks = n_total == 0 ? 0 : (n_total + chunk_elems - 1) / chunk_elems;
+  uint16_t* pout = static_cast<uint16_t*>(param_bf16_out);
+
+  CU(cudaEventRecord(ctx->ev_begin, ctx->s_compute));
+  CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_begin, 0));
+  for (int64_t c = 0; c < nchunks; ++c) {
+    const int slot = (int)(c % nbuf);
+    const int64_t off = c * chunk_elems;
+    const int64_t len = n_total - off < chunk_elems ? n_total - off : chunk_elems;
+    float* sw = ctx->slots + (size_t)slot * cap;
+    // copy-in: the slot must have been read by the cast of chunk c - nbuf
+    if (c >= nbuf) CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_free[slot], 0));
+    if (stats && c == 0) CU(cudaEventRecord(ctx->ev_in_first, ctx->s_in));
+    CU(cudaMemcpyAsync(sw, host_master + off, (size_t)len * sizeof(float),
+                       cudaMemcpyHostToDevice, ctx->s_in));
+    if (stats && c == nchunks - 1) CU(cudaEventRecord(ctx->ev_in_last, ctx->s_in));
+    CU(cudaEventRecord(ctx->ev_loaded[slot], ctx->s_in));
+    // cast
+    CU(cudaStreamWaitEvent(ctx->s_compute, ctx->ev_loaded[slot], 0));
+    const unsigned blocks = (unsigned)((len + 8 * kCastThreads - 1) / (8 * kCastThreads));
+    cast_master_to_bf16_kernel<<<blocks, kCastThreads, 0, ctx->s_compute>>>(sw, len, pout + off);
+    ctx->launches += 1;
+    CU(cudaGetLastError());
+    CU(cudaEventRecord(ctx->ev_free[slot], ctx->s_compute));
+  }
+  CU(cudaEventRecord(ctx->ev_end, ctx->s_compute));
+  rc = bounded_event_wait(ctx, ctx->ev_end, kWaitSeconds);
+  if (rc != SLIDEDP_OK) return rc;
+  rc = bounded_stream_wait(ctx, ctx->s_in, kWaitSeconds);
+  if (rc != SLIDEDP_OK) return rc;
+  if (stats) {
+    float ms = 0.f;
+    CU(cudaEventElapsedTime(&ms, ctx->ev_begin, ctx->ev_end));
+    stats->ms_total = ms;
+    stats->chunks = nchunks;
+    if (nchunks > 0) {
+      CU(cudaEventElapsedTime(&ms, ctx->ev_in_first, ctx->ev_in_last));
+      stats->ms_h2d = ms;
+      if (ms > 0) stats->gbs_h2d = 4.0 * (double)n_total / (ms * 1e6);
+    }
+  }
+  return SLIDEDP_OK;
+}
+
+int slidedp_model_stream_step(int64_t n_total, int R, int64_t chunk_elems, int nbuf,
+                              const slidedp_rates* rates, double* lower_bound_ms,
+                              double* predicted_ms) {
+  if (n_total < 0 || R < 1 || R > SLIDEDP_MAX_RANKS || chunk_elems <= 0 || nbuf < 1 || !rates ||
+      !lower_bound_ms || !predicted_ms)
+    return SLIDEDP_ERR_INVALID_ARG;
+  if (!(rates->h2d_gbs > 0.0) || !(rates->d2h_gbs > 0.0) || !(rates->update_gparams_s > 0.0) ||
+      !(rates->norm_gbs >= 0.0) || !(rates->per_copy_us >= 0.0))
+    return SLIDEDP_ERR_INVALID_ARG;
+  const int64_t nchunks = n_total == 0 ? 0 : (n_total + chunk_elems - 1) / chunk_elems;
+  const double norm_ms =
+      rates->norm_gbs > 0.0 ? 2.0 * R * (double)n_total / (rates->norm_gbs * 1e6) : 0.0;
+  const double copy_fixed_ms = 3.0 * rates->per_copy_us * 1e-3;
+  // resource demand: W_j / beta_j per lane
+  const double in_ms = 12.0 * (double)n_total / (rates->h2d_gbs * 1e6) + nchunks * copy_fixed_ms;
+  const double out_ms = 12.0 * (double)n_total / (rates->d2h_gbs * 1e6) + nchunks * copy_fixed_ms;
+  const double compute_ms = norm_ms + (double)n_total / (rates->update_gparams_s * 1e6);
+  double bound = in_ms > out_ms ? in_ms : out_ms;
+  if (compute_ms > bound) bound = compute_ms;
+  *lower_bound_ms = bound;
+  // execution dependencies: completion times, chunk by chunk; the last nbuf copy-outs are kept
+  std::vector<double> out_done((size_t)nbuf, 0.0);
+  double f_in = 0.0, f_k = norm_ms, f_out = 0.0;
+  for (int64_t c = 0; c < nchunks; ++c) {
+    const int64_t len = n_total - c * chunk_elems < chunk_elems ? n_total - c * chunk_elems
+                                                                 : chunk_elems;
+    const double d_in = 12.0 * (double)len / (rates->h2d_gbs * 1e6) + copy_fixed_ms;
+    const double d_k = (double)len / (rates->update_gparams_s * 1e6);
+    const double d_out = 12.0 * (double)len / (rates->d2h_gbs * 1e6) + copy_fixed_ms;
+    const double slot_free = c >= nbuf ? out_done[(size_t)(c % nbuf)] : 0.0;
+    f_in = d_in + (f_in > slot_free ? f_in : slot_free);
+    f_k = d_k + (f_k > f_in ? f_k : f_in);
+    f_out = d_out + (f_out > f_k ? f_out : f_k);
+    out_done[(size_t)(c % nbuf)] = f_out;
+  }
+  *predicted_ms = f_out > f_k ? f_out : f_k;
   return SLIDEDP_OK;
 }
 
@@ -649,10 +761,7 @@ int slidedp_grad_norm_noalloc(const void* const* grads_bf16, int R, int64_t n, d
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
   if (ntiles > 0) {
-    int sms = 148;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int64_t max_blocks = (int64_t)sms * 8;
-    const unsigned blocks = (unsigned)(ntiles < max_blocks ? ntiles : max_blocks);
+    const unsigned blocks = (unsigned)ntiles;
     const float inv = (float)inv_R;
     switch (R) {
       case 1: grad_sumsq_tiles_kernel<1><<<blocks, kNormThreads, 0, st>>>(gp, R, n, inv, scratch); break;

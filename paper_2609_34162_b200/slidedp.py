@@ -86,6 +86,9 @@ _lib.slidedp_stream_step.restype = ctypes.c_int
 _lib.slidedp_stream_step.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp, _vp,
                                      ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                      ctypes.POINTER(_HParams), ctypes.POINTER(_Stats)]
+_lib.slidedp_deliver_params.restype = ctypes.c_int
+_lib.slidedp_deliver_params.argtypes = [_vp, _vp, ctypes.c_int64, _vp, ctypes.c_int64, ctypes.c_int,
+                                        ctypes.POINTER(_Stats)]
 _lib.slidedp_link_probe.restype = ctypes.c_int
 _lib.slidedp_link_probe.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_size_t, ctypes.c_size_t,
                                     ctypes.c_int, ctypes.POINTER(ctypes.c_double)]
@@ -94,6 +97,18 @@ _lib.slidedp_grad_norm_noalloc.argtypes = [_pp, ctypes.c_int, ctypes.c_int64, ct
                                            ctypes.c_double, _vp, _vp]
 _lib.slidedp_kernel_launches.restype = ctypes.c_int64
 _lib.slidedp_kernel_launches.argtypes = [_vp]
+
+
+class _Rates(ctypes.Structure):
+    _fields_ = [("h2d_gbs", ctypes.c_double), ("d2h_gbs", ctypes.c_double),
+                ("update_gparams_s", ctypes.c_double), ("norm_gbs", ctypes.c_double),
+                ("per_copy_us", ctypes.c_double)]
+
+
+_lib.slidedp_model_stream_step.restype = ctypes.c_int
+_lib.slidedp_model_stream_step.argtypes = [ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_int,
+                                           ctypes.POINTER(_Rates), ctypes.POINTER(ctypes.c_double),
+                                           ctypes.POINTER(ctypes.c_double)]
 
 
 class SlideDPError(RuntimeError):
@@ -210,12 +225,35 @@ class Context:
             return None
         return {f: getattr(st, f) for f, _ in _Stats._fields_ if f != "reserved"}
 
+    def slidedp_deliver_params(self, host_master, n_total: int, param_bf16_out, chunk_elems: int,
+                               nbuf: int, want_stats: bool = True):
+        st = _Stats()
+        self._check(_lib.slidedp_deliver_params(
+            self._h, _ptr(host_master), n_total, _ptr(param_bf16_out), chunk_elems, nbuf,
+            ctypes.byref(st) if want_stats else None))
+        if not want_stats:
+            return None
+        return {f: getattr(st, f) for f in ("ms_total", "ms_h2d", "gbs_h2d", "chunks")}
+
     def slidedp_link_probe(self, host_a, host_b, dev_a, dev_b, nbytes: int, copy_bytes: int,
                            reps: int = 3):
         out = (ctypes.c_double * 4)()
         self._check(_lib.slidedp_link_probe(self._h, _ptr(host_a), _ptr(host_b), _ptr(dev_a),
                                             _ptr(dev_b), nbytes, copy_bytes, reps, out))
         return {"h2d": out[0], "d2h": out[1], "h2d_bidir": out[2], "d2h_bidir": out[3]}
+
+
+def slidedp_model_stream_step(n_total: int, R: int, chunk_elems: int, nbuf: int, h2d_gbs: float,
+                              d2h_gbs: float, update_gparams_s: float, norm_gbs: float = 0.0,
+                              per_copy_us: float = 0.0):
+    """(lower_bound_ms, predicted_ms) of a host-resident step from measured rates."""
+    r = _Rates(h2d_gbs, d2h_gbs, update_gparams_s, norm_gbs, per_copy_us)
+    lo, pred = ctypes.c_double(), ctypes.c_double()
+    rc = _lib.slidedp_model_stream_step(n_total, R, chunk_elems, nbuf, ctypes.byref(r),
+                                        ctypes.byref(lo), ctypes.byref(pred))
+    if rc != OK:
+        raise SlideDPError(rc)
+    return lo.value, pred.value
 
 
 def slidedp_create(device: int = 0, gpu_budget_bytes: int = 0) -> Context:

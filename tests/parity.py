@@ -25,23 +25,22 @@ def f32(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().contiguous().numpy()
 
 
-def fp32_violations(got: np.ndarray, want: np.ndarray, block: int = 1 << 24):
-    """(count outside tolerance, worst ratio |x-y| / allowed), streaming to bound memory."""
+def fp32_violations(got: np.ndarray, want: np.ndarray, block: int = 1 << 26):
+    """(count outside tolerance, worst ratio |x-y| / allowed). Streams in blocks and uses torch's
+    threaded CPU ops so that multi-billion-element states compare in seconds."""
     assert got.shape == want.shape and got.dtype == np.float32 and want.dtype == np.float32
     bad, worst = 0, 0.0
     for lo in range(0, got.size, block):
-        x = got[lo:lo + block].astype(np.float64)
-        y = want[lo:lo + block].astype(np.float64)
-        allowed = np.maximum(FP32_RTOL * np.abs(y), FP32_ATOL)
-        err = np.abs(x - y)
-        both_nan = np.isnan(x) & np.isnan(y)
-        err[both_nan] = 0.0
-        err[np.isnan(err)] = np.inf
-        same_inf = np.isinf(x) & (x == y)
-        err[same_inf] = 0.0
+        x = torch.from_numpy(got[lo:lo + block]).double()
+        y = torch.from_numpy(want[lo:lo + block]).double()
+        allowed = torch.clamp(FP32_RTOL * y.abs(), min=FP32_ATOL)
+        err = (x - y).abs()
+        same_special = (torch.isnan(x) & torch.isnan(y)) | (torch.isinf(x) & (x == y))
+        err = torch.where(same_special, torch.zeros_like(err), err)
+        err = torch.where(torch.isnan(err), torch.full_like(err, float("inf")), err)
         ratio = err / allowed
         bad += int((ratio > 1.0).sum())
-        if ratio.size:
+        if ratio.numel():
             worst = max(worst, float(ratio.max()))
     return bad, worst
 
@@ -52,19 +51,25 @@ def assert_fp32_close(name: str, got: np.ndarray, want: np.ndarray):
     return worst
 
 
-def _bf16_line(bits: np.ndarray) -> np.ndarray:
+def _bf16_line(bits: torch.Tensor) -> torch.Tensor:
     """Monotone integer line over BF16 patterns (so that adjacent values differ by 1)."""
-    i = bits.astype(np.int32)
-    return np.where(i & 0x8000, -(i & 0x7FFF), i)
+    i = bits.to(torch.int32) & 0xFFFF
+    return torch.where((i & 0x8000) != 0, -(i & 0x7FFF), i)
 
 
-def bf16_mismatch(got: np.ndarray, want: np.ndarray):
+def bf16_mismatch(got: np.ndarray, want: np.ndarray, block: int = 1 << 26):
     """(max ulp distance, fraction of elements that differ)."""
     assert got.shape == want.shape and got.dtype == np.uint16 and want.dtype == np.uint16
     if got.size == 0:
         return 0, 0.0
-    d = np.abs(_bf16_line(got) - _bf16_line(want))
-    return int(d.max()), float((d != 0).sum()) / got.size
+    worst, differ = 0, 0
+    for lo in range(0, got.size, block):
+        a = torch.from_numpy(got[lo:lo + block].view(np.int16))
+        b = torch.from_numpy(want[lo:lo + block].view(np.int16))
+        d = (_bf16_line(a) - _bf16_line(b)).abs()
+        worst = max(worst, int(d.max()))
+        differ += int((d != 0).sum())
+    return worst, differ / got.size
 
 
 def assert_bf16_close(name: str, got: np.ndarray, want: np.ndarray):

@@ -272,7 +272,7 @@ def test_indices_beyond_2_to_31(ctx, sd):
     m = w * 0.01
     v = w * w * 1e-3
     p = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
-    slices = [(0, 1 << 20), ((1 << 31) - (1 << 19), (1 << 31) + (1 << 19)), (n - (1 << 20), n)]
+    slices = [(0, 1 << 20), ((1 << 31) - (1 << 19), (1 << 31) + 2048), (n - (1 << 20), n)]
     before = [[parity.f32(t[a:b]).copy() for t in (w, m, v)] for a, b in slices]
     kw = dict(ADAM, inv_R=1.0, max_norm=1.0, step=11)
     ctx.slidedp_grad_norm([g], n, 1.0, True)

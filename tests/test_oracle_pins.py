@@ -415,3 +415,18 @@ def test_multi_step_equals_repeated_single_steps_and_empty_chunk():
     z = np.zeros(0, np.float32)
     assert oracle.step([np.zeros(0, np.uint16)] * 2, z, z.copy(), z.copy(),
                        np.zeros(0, np.uint16), HParams(inv_R=0.5, max_norm=1.0)) == (0.0, 1.0)
+
+
+# -------------------------------------------------------------- parameter delivery cast
+def test_delivery_cast_matches_torch_cast_and_keeps_specials():
+    rng = np.random.default_rng(15)
+    x = (rng.standard_normal(200_000) * 0.02).astype(np.float32)
+    x[:8] = [0.0, -0.0, np.inf, -np.inf, 1.00390625, 1.01171875, 1e-40, -3.4e38]
+    #        ties: 1 + 2^-8 -> 1.0 (even), 1 + 3*2^-8 -> 1 + 2^-6 (even); subnormal; near max
+    got = oracle.cast_master_to_bf16(x)
+    assert np.array_equal(got, bf16_bits(x))
+    assert got[4] == 0x3F80 and got[5] == 0x3F82 and got[2] == 0x7F80 and got[3] == 0xFF80
+    assert got[1] == 0x8000 and got[7] == 0xFF80            # -3.4e38 rounds to -inf in BF16
+    nan = oracle.cast_master_to_bf16(np.array([np.nan], np.float32))[0]
+    assert (nan & 0x7F80) == 0x7F80 and (nan & 0x7F) != 0
+    assert oracle.cast_master_to_bf16(np.zeros(0, np.float32)).size == 0

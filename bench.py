@@ -461,7 +461,24 @@ def run_sweep(args):
         norm_ms.append(e0.elapsed_time(e1))
     ms = statistics.mean(step_ms[2:])
     nm = statistics.mean(norm_ms[2:])
+    # the same step with the layers enqueued back to back (one wait at the end)
+    async_ms = []
+    for t in range(wl.steps + 1, wl.steps + 6):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for l in range(L):
+            ctx.slidedp_grad_norm(grads[l], nl, 1.0 / R, l == 0)
+        ctx.slidedp_grad_norm_finish(wl.max_norm)
+        torch.cuda.synchronize()
+        for l in range(L):
+            ctx.slidedp_stream_step_async(grads[l], nl, *state[l], ps[l], ce, 3, hp(wl, t),
+                                          norm_ready=True)
+        ctx.slidedp_stream_wait()
+        async_ms.append((time.perf_counter() - t0) * 1e3)
+    ams = statistics.mean(async_ms[1:])
     out["qwen3_14b_8layers_host"] = {
+        "async_layers": {"ms_per_step": ams, "g_params_per_s": wl.numel / ams / 1e6,
+                         "link_gbs_each_way": 12.0 * wl.numel / (ams * 1e6)},
         "params": wl.numel, "R": R, "layers": L, "steps": wl.steps, "chunk_mib": 64, "nbuf": 3,
         "ms_per_step": ms, "g_params_per_s": wl.numel / ms / 1e6,
         "link_gbs_each_way": 12.0 * wl.numel / (ms * 1e6),

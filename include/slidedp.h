@@ -166,6 +166,19 @@ SLIDEDP_API int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_b
                         void* param_bf16_out, int64_t chunk_elems, int nbuf, int norm_ready,
                         const slidedp_hparams* hp, slidedp_stats* stats);
 
+/* The same step without the final wait, for callers that stream several layers back to back
+ * (Sec. 3.3: completed layers release their updates while other work continues). The call only
+ * enqueues; consecutive calls share the slot ring, so the copy-out of one layer's last chunk runs
+ * beside the copy-in of the next layer's first chunk instead of draining the pipeline per
+ * layer. The host arrays, gradients and output must stay valid, and the context's clip
+ * coefficient unchanged, until slidedp_stream_wait returns; that call waits (bounded) for
+ * everything queued. A call whose slot layout differs (chunk_elems, nbuf) first drains. */
+SLIDEDP_API int slidedp_stream_step_async(slidedp_ctx* ctx, const void* const* grads_bf16, int R,
+                              int64_t n_total, float* host_master, float* host_m, float* host_v,
+                              void* param_bf16_out, int64_t chunk_elems, int nbuf, int norm_ready,
+                              const slidedp_hparams* hp);
+SLIDEDP_API int slidedp_stream_wait(slidedp_ctx* ctx);
+
 /* ---- parameter delivery: BF16 copy of a host-resident FP32 master -------------------------
  *
  * The step BEFORE the update path (paper Sec. 3.3 "Overlap within a layer": on parameter

@@ -86,6 +86,12 @@ _lib.slidedp_stream_step.restype = ctypes.c_int
 _lib.slidedp_stream_step.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp, _vp,
                                      ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                      ctypes.POINTER(_HParams), ctypes.POINTER(_Stats)]
+_lib.slidedp_stream_step_async.restype = ctypes.c_int
+_lib.slidedp_stream_step_async.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp, _vp,
+                                           ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                           ctypes.POINTER(_HParams)]
+_lib.slidedp_stream_wait.restype = ctypes.c_int
+_lib.slidedp_stream_wait.argtypes = [_vp]
 _lib.slidedp_deliver_params.restype = ctypes.c_int
 _lib.slidedp_deliver_params.argtypes = [_vp, _vp, ctypes.c_int64, _vp, ctypes.c_int64, ctypes.c_int,
                                         ctypes.POINTER(_Stats)]
@@ -224,6 +230,18 @@ class Context:
         if not want_stats:
             return None
         return {f: getattr(st, f) for f, _ in _Stats._fields_ if f != "reserved"}
+
+    def slidedp_stream_step_async(self, grads, n_total: int, host_master, host_m, host_v,
+                                  param_bf16_out, chunk_elems: int, nbuf: int, hp: HParams,
+                                  norm_ready: bool = False) -> None:
+        c = hp._c()
+        self._check(_lib.slidedp_stream_step_async(
+            self._h, _grad_array(grads), len(grads), n_total, _ptr(host_master), _ptr(host_m),
+            _ptr(host_v), _ptr(param_bf16_out), chunk_elems, nbuf, int(norm_ready),
+            ctypes.byref(c)))
+
+    def slidedp_stream_wait(self) -> None:
+        self._check(_lib.slidedp_stream_wait(self._h))
 
     def slidedp_deliver_params(self, host_master, n_total: int, param_bf16_out, chunk_elems: int,
                                nbuf: int, want_stats: bool = True):

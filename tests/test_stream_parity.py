@@ -201,3 +201,48 @@ def test_stream_step_argument_errors(ctx, sd):
         small.slidedp_destroy()
     st = call(g, 0, hw, hm, hv, p, 1024, 3, hp)
     assert st["chunks"] == 0
+
+
+def test_async_layers_share_the_slot_ring_and_match_the_synchronous_step(ctx, sd):
+    """Several layers enqueued back to back with slidedp_stream_step_async (one wait at the
+    end), with layer sizes that leave short last chunks and a change of chunk size in between,
+    give bit-identical state to one synchronous call per layer."""
+    wl = W.scaled(W.CONFIGS["qwen3_14b_8layers_host"], 64)
+    L, R, nl = 4, wl.R, wl.layer_numel
+    kw = dict(inv_R=1.0 / R, max_norm=wl.max_norm, step=3, **wl.hparams)
+    dg = [[W.rank_gradient(wl, r, step=3, layer=l, device="cuda") for r in range(R)]
+          for l in range(L)]
+    init = [[parity.f32(W.master_weights(wl, layer=l, device="cuda")),
+             np.full(nl, 1e-4, np.float32), np.full(nl, 1e-7, np.float32)] for l in range(L)]
+    for l in range(L):
+        ctx.slidedp_grad_norm(dg[l], nl, kw["inv_R"], l == 0)
+    ctx.slidedp_grad_norm_finish(wl.max_norm, fetch=True)
+    chunks = [1 << 19, 1 << 19, 3 * (1 << 17), 1 << 19]          # layer 2 forces a re-layout
+
+    def run(asynchronous):
+        host = [[pinned(a) for a in init[l]] for l in range(L)]
+        dp = [torch.zeros(nl, dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+        for l in range(L):
+            args = (dg[l], nl, host[l][0], host[l][1], host[l][2], dp[l], chunks[l], 3,
+                    sd.HParams(**kw))
+            if asynchronous:
+                ctx.slidedp_stream_step_async(*args, norm_ready=True)
+            else:
+                ctx.slidedp_stream_step(*args, norm_ready=True)
+        if asynchronous:
+            ctx.slidedp_stream_wait()
+        return [[h.numpy().copy() for h in host[l]] + [parity.u16(dp[l])] for l in range(L)]
+
+    sync, asyn = run(False), run(True)
+    for l in range(L):
+        for a, b in zip(sync[l], asyn[l]):
+            assert np.array_equal(a, b)
+    # and a delivery right after queued async work sees the finished master
+    host = [pinned(a) for a in init[0]]
+    dp = torch.zeros(nl, dtype=torch.bfloat16, device="cuda")
+    ctx.slidedp_stream_step_async(dg[0], nl, host[0], host[1], host[2], dp, 1 << 19, 3,
+                                  sd.HParams(**kw), norm_ready=True)
+    out = torch.zeros(nl, dtype=torch.bfloat16, device="cuda")
+    ctx.slidedp_deliver_params(host[0], nl, out, 1 << 18, 2)
+    assert np.array_equal(parity.u16(out), parity.u16(dp))
+    ctx.slidedp_stream_wait()

@@ -103,37 +103,33 @@ __device__ __forceinline__ void adamw_element(float gbar, float& w, float& m, fl
 // is what hides the FP64 dependency chains behind the loads of the other warps. Measured
 // on B200: 6.58 TB/s against 5.6 TB/s for the eight-per-thread form and 6.4 TB/s for a
 // bulk-copy (TMA) shared-memory ring.
-// R_T > 0: rank count known at compile time (loads fully unrolled). R_T == 0: runtime R.
-template <int R_T>
+// R is a template parameter (one instantiation per rank count 1..16): the R loads and the
+// left-to-right FP32 adds are fully unrolled.
+template <int R>
 __global__ void __launch_bounds__(kUpdateThreads, 4)
-reduce_adamw_kernel(GradPtrs gp, int R_rt, int64_t n, float* __restrict__ master,
+reduce_adamw_kernel(GradPtrs gp, int64_t n, float* __restrict__ master,
                     float* __restrict__ mom1, float* __restrict__ mom2,
                     uint16_t* __restrict__ param_out, UpdateConsts k,
                     const double* __restrict__ clip_coef) {
-  constexpr int RMAX = R_T > 0 ? R_T : kMaxRanks;
-  const int R = R_T > 0 ? R_T : R_rt;
   const int64_t base = ((int64_t)blockIdx.x * kUpdateThreads + threadIdx.x) * kVec;
   if (base >= n) return;
   const double c = clip_coef ? *clip_coef : 1.0;
   const double k1 = k.omb1 * c, k2 = k.omb2 * c * c;
 
   if (base + kVec <= n) {
-    uint2 graw[RMAX];
+    uint2 graw[R];
 #pragma unroll
-    for (int r = 0; r < RMAX; ++r)
-      if (r < R) graw[r] = __ldcs(reinterpret_cast<const uint2*>(gp.p[r] + base));
+    for (int r = 0; r < R; ++r) graw[r] = __ldcs(reinterpret_cast<const uint2*>(gp.p[r] + base));
     uint4 wq = ld_stream(master + base);
     uint4 mq = ld_stream(mom1 + base);
     uint4 vq = ld_stream(mom2 + base);
     float s[kVec] = {bf16_lo(graw[0].x), bf16_hi(graw[0].x), bf16_lo(graw[0].y), bf16_hi(graw[0].y)};
 #pragma unroll
-    for (int r = 1; r < RMAX; ++r) {
-      if (r < R) {
-        s[0] = __fadd_rn(s[0], bf16_lo(graw[r].x));
-        s[1] = __fadd_rn(s[1], bf16_hi(graw[r].x));
-        s[2] = __fadd_rn(s[2], bf16_lo(graw[r].y));
-        s[3] = __fadd_rn(s[3], bf16_hi(graw[r].y));
-      }
+    for (int r = 1; r < R; ++r) {
+      s[0] = __fadd_rn(s[0], bf16_lo(graw[r].x));
+      s[1] = __fadd_rn(s[1], bf16_hi(graw[r].x));
+      s[2] = __fadd_rn(s[2], bf16_lo(graw[r].y));
+      s[3] = __fadd_rn(s[3], bf16_hi(graw[r].y));
     }
     float* wf = reinterpret_cast<float*>(&wq);
     float* mf = reinterpret_cast<float*>(&mq);
@@ -170,11 +166,9 @@ reduce_adamw_kernel(GradPtrs gp, int R_rt, int64_t n, float* __restrict__ master
 // a tile's partial does not depend on which block computes it or on the grid size.
 // Launched with one block per tile; the loads of UNROLL iterations are in flight together
 // (measured best: 2 at R = 4, 1 at R = 8, where more unrolling costs occupancy).
-template <int R_T, int UNROLL = (R_T == 0 || R_T >= 8) ? 1 : (R_T >= 4 ? 2 : 4)>
+template <int R, int UNROLL = (R >= 6) ? 1 : (R >= 3 ? 2 : 4)>
 __global__ void __launch_bounds__(kNormThreads)
-grad_sumsq_tiles_kernel(GradPtrs gp, int R_rt, int64_t n, float inv_R,
-                        double* __restrict__ partials) {
-  const int R = R_T > 0 ? R_T : R_rt;
+grad_sumsq_tiles_kernel(GradPtrs gp, int64_t n, float inv_R, double* __restrict__ partials) {
   __shared__ double warp_sum[kNormThreads / 32];
   const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
@@ -185,24 +179,21 @@ grad_sumsq_tiles_kernel(GradPtrs gp, int R_rt, int64_t n, float inv_R,
       const int64_t e = tbase + (int64_t)it * (kNormThreads * kNormVec);
       float s[kNormVec];
       if (e + kNormVec <= n) {
-        uint4 graw[R_T > 0 ? R_T : kMaxRanks];
+        uint4 graw[R];
 #pragma unroll
-        for (int r = 0; r < (R_T > 0 ? R_T : kMaxRanks); ++r)
-          if (r < R) graw[r] = ld_stream(gp.p[r] + e);
+        for (int r = 0; r < R; ++r) graw[r] = ld_stream(gp.p[r] + e);
         {
           const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[0]);
 #pragma unroll
           for (int j = 0; j < 4; ++j) { s[2 * j] = bf16_lo(x[j]); s[2 * j + 1] = bf16_hi(x[j]); }
         }
 #pragma unroll
-        for (int r = 1; r < (R_T > 0 ? R_T : kMaxRanks); ++r) {
-          if (r < R) {
-            const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[r]);
+        for (int r = 1; r < R; ++r) {
+          const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[r]);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              s[2 * j] = __fadd_rn(s[2 * j], bf16_lo(x[j]));
-              s[2 * j + 1] = __fadd_rn(s[2 * j + 1], bf16_hi(x[j]));
-            }
+          for (int j = 0; j < 4; ++j) {
+            s[2 * j] = __fadd_rn(s[2 * j], bf16_lo(x[j]));
+            s[2 * j + 1] = __fadd_rn(s[2 * j + 1], bf16_hi(x[j]));
           }
         }
       } else {

@@ -91,6 +91,19 @@ def test_odd_sizes_all_rank_counts(ctx, sd, n, R):
         assert_parity(f"n={n} R={R} clip={clip}", got, want, clip)
 
 
+@pytest.mark.parametrize("R", list(range(1, 17)))
+def test_every_rank_count_has_its_own_kernel(ctx, sd, R):
+    """R = 1..16 each run a kernel with the rank loop unrolled; wide exponent spread between
+    ranks so that the left-to-right order of the FP32 adds shows in the result."""
+    n = (1 << 16) + 5
+    g = torch.Generator().manual_seed(4000 + R)
+    scale = 2.0 ** torch.randint(-12, 1, (R, n), generator=g).float()
+    grads = [(torch.randn(n, generator=g) * 1e-2 * scale[r]).to(torch.bfloat16) for r in range(R)]
+    _, w, m, v = random_case(n, 1, seed=R)
+    got, want = run_both(ctx, sd, grads, w, m, v, dict(ADAM, step=4), 0.3)
+    assert_parity(f"R={R}", got, want, 0.3)
+
+
 def test_empty_chunk_is_a_no_op(ctx, sd):
     hp_g, _ = hp_pair(sd, inv_R=0.5, step=1, **ADAM)
     g = [torch.zeros(8, dtype=torch.bfloat16, device="cuda") for _ in range(2)]

@@ -307,3 +307,40 @@ def test_indices_beyond_2_to_31(ctx, sd):
         parity.assert_bf16_close(tag + "/param_bf16", parity.u16(p[a:b]), op)
     # nothing outside the chunk was touched and every element inside was written
     assert int((p == 0).sum()) < n // 1000
+
+
+@pytest.mark.parametrize("n", [1, 3, 4, 5, 1021, 1024, 1027, 16384, 16385, 65536 + 7])
+def test_guard_bands_around_every_buffer_stay_intact(ctx, sd, n):
+    """Every output (and input) sits between 64-element canary bands; after the norm, the update
+    and the delivery cast, the bands are unchanged and every element inside was written once."""
+    R, pad = 3, 64
+    gen = torch.Generator(device="cuda").manual_seed(n)
+
+    def banded(dtype, fill):
+        t = torch.full((n + 2 * pad,), fill, dtype=dtype, device="cuda")
+        return t, t[pad:pad + n]
+
+    gfull, grads = zip(*[banded(torch.bfloat16, 123.0) for _ in range(R)])
+    for g in grads:
+        g.copy_((torch.randn(n, generator=gen, device="cuda") * 1e-3).to(torch.bfloat16))
+    wfull, w = banded(torch.float32, -7.0)
+    mfull, m = banded(torch.float32, -7.0)
+    vfull, v = banded(torch.float32, -7.0)
+    pfull, p = banded(torch.bfloat16, -7.0)
+    w.copy_(torch.randn(n, generator=gen, device="cuda") * 0.02); m.zero_(); v.zero_()
+    snap = [t.clone() for t in gfull]
+    ctx.slidedp_grad_norm(list(grads), n, 1.0 / R, True)
+    ctx.slidedp_grad_norm_finish(0.01)
+    ctx.slidedp_reduce_adamw_chunk(list(grads), n, w, m, v, p, sd.HParams(inv_R=1.0 / R, max_norm=0.01,
+                                                                           step=1))
+    torch.cuda.synchronize()
+    for full, fill in ((wfull, -7.0), (mfull, -7.0), (vfull, -7.0), (pfull, -7.0)):
+        assert torch.all(full[:pad] == fill) and torch.all(full[pad + n:] == fill)
+    assert all(torch.equal(a, b) for a, b in zip(snap, gfull))          # gradients are read-only
+    assert torch.all(p.float() != -7.0) and torch.all(v >= 0) and torch.all(m.abs() < 1.0)
+    # delivery cast into a banded output
+    host = torch.empty(n, pin_memory=True); host.copy_(w)
+    pfull.fill_(-7.0)
+    ctx.slidedp_deliver_params(host, n, p, 8, 2)
+    assert torch.all(pfull[:pad] == -7.0) and torch.all(pfull[pad + n:] == -7.0)
+    assert torch.equal(p, w.to(torch.bfloat16))

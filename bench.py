@@ -32,9 +32,9 @@ UNIT = "G-params/s"
 WORKLOAD = "qwen3_8b_layer"
 HOST_WORKLOAD = "qwen3_14b_layer_host"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per parameter of the fused update kernel, from
-# the ncu capture summarised in profiles/reduce_adamw_kernel_R4_50M_params.md (50 M-parameter case,
-# scaled to a full launch by the parameter count).
+# dram__bytes_read.sum + dram__bytes_write.sum per parameter of the fused update kernel, from an
+# ncu capture of a 50 M-parameter, R = 4 launch (a full-size launch is above the size an ncu
+# capture should hold); scaled to a full launch by the parameter count.
 NCU_TRAFFIC_BYTES_PER_PARAM = 32.92
 
 

@@ -13,7 +13,7 @@ namespace slidedp {
 
 constexpr int kMaxRanks = 16;
 constexpr int kVec = 4;                 // parameters per thread in the update kernel
-constexpr int kUpdateThreads = 256;
+constexpr int kUpdateThreads = 128;
 constexpr int kNormVec = 8;             // elements per thread per load in the norm kernel
 constexpr int kNormThreads = 256;
 constexpr int kNormIters = 8;
@@ -72,23 +72,31 @@ __device__ __forceinline__ double rcp_seed(double x) {
 
 // One parameter's AdamW update in FP64 from the FP32 state. k1 = (1-beta1) c and
 // k2 = (1-beta2) c^2 carry the clip coefficient c.
+//
+// The common path has no FP64 compares: sqrt(v1) and m1/d come from the hardware seeds plus
+// one Newton step each (~1e-12 relative). v1 == 0 (zero gradient on zero state) is caught by an
+// integer test of the double's high word, because the rsqrt seed of 0 is +inf. Everything else
+// that the seeds cannot carry (v1 = +inf, d = 0 when eps = 0, NaN or inf operands) makes the
+// result non-finite, and only then the update is redone with IEEE sqrt and division, so those
+// cases follow the plain formulas exactly (e.g. v1 = inf gives u = 0, a finite decay-only step).
 __device__ __forceinline__ void adamw_element(float gbar, float& w, float& m, float& v,
                                               const UpdateConsts& k, double k1, double k2) {
   const double g = (double)gbar;
+  const double w0 = (double)w;
   const double m1 = fma(k.beta1, (double)m, k1 * g);
   const double v1 = fma(k.beta2, (double)v, k2 * (g * g));     // g*g is exact in double
-  // s = sqrt(v1): seed, then one Newton step on the root itself.
-  const double r = v1 > 0.0 ? rsqrt_seed(v1) : 0.0;
+  const double r = (__double2hiint(v1) == 0) ? 0.0 : rsqrt_seed(v1);
   double s = v1 * r;
-  s = fma(fma(-s, s, v1), 0.5 * r, s);
-  if (!(v1 < 1.7976931348623157e308)) s = v1;                  // +inf and NaN pass through
+  s = fma(fma(-s, s, v1), 0.5 * r, s);                         // s = sqrt(v1)
   const double d = fma(s, k.rsqrt_bc2, k.eps);                 // sqrt(v1/bc2) + eps
-  // q = m1 / d: seed reciprocal, one correction of the quotient.
   const double rc = rcp_seed(d);
   double q = m1 * rc;
-  q = fma(fma(-q, d, m1), rc, q);
-  if (!(d > 0.0) || !(d < 1.7976931348623157e308)) q = m1 / d; // 0, inf, NaN: IEEE division
-  const double w1 = fma(k.neg_lr_over_bc1, q, k.decay * (double)w);
+  q = fma(fma(-q, d, m1), rc, q);                              // q = m1 / d
+  double w1 = fma(k.neg_lr_over_bc1, q, k.decay * w0);
+  if ((__double2hiint(w1) & 0x7ff00000) == 0x7ff00000) {       // inf or NaN: rare, exact path
+    const double d2 = fma(sqrt(v1), k.rsqrt_bc2, k.eps);
+    w1 = fma(k.neg_lr_over_bc1, m1 / d2, k.decay * w0);
+  }
   m = __double2float_rn(m1);
   v = __double2float_rn(v1);
   w = __double2float_rn(w1);
@@ -99,14 +107,14 @@ __device__ __forceinline__ void adamw_element(float gbar, float& w, float& m, fl
 // One thread owns kVec = 4 consecutive parameters: one 8-byte BF16 load per rank, one
 // 16-byte load per FP32 array, all issued before the first use, then the FP64 update in
 // registers and one store per output. Four parameters (not eight) per thread keeps the
-// kernel at 64 registers, so four 256-thread blocks (32 warps) stay resident per SM; that
+// kernel at 64 registers, so eight 128-thread blocks (32 warps) stay resident per SM; that
 // is what hides the FP64 dependency chains behind the loads of the other warps. Measured
-// on B200: 6.58 TB/s against 5.6 TB/s for the eight-per-thread form and 6.4 TB/s for a
-// bulk-copy (TMA) shared-memory ring.
+// on B200 at R = 4: 6.8-6.9 TB/s against 5.6 TB/s for the eight-per-thread form and 6.4 TB/s
+// for a bulk-copy (TMA) shared-memory ring.
 // R is a template parameter (one instantiation per rank count 1..16): the R loads and the
 // left-to-right FP32 adds are fully unrolled.
 template <int R>
-__global__ void __launch_bounds__(kUpdateThreads, 4)
+__global__ void __launch_bounds__(kUpdateThreads, 8)
 reduce_adamw_kernel(GradPtrs gp, int64_t n, float* __restrict__ master,
                     float* __restrict__ mom1, float* __restrict__ mom2,
                     uint16_t* __restrict__ param_out, UpdateConsts k,

@@ -48,6 +48,8 @@ def fp32_violations(got: np.ndarray, want: np.ndarray, block: int = 1 << 26):
 def assert_fp32_close(name: str, got: np.ndarray, want: np.ndarray):
     bad, worst = fp32_violations(got, want)
     assert bad == 0, f"{name}: {bad} of {got.size} elements outside tolerance (worst {worst:.3g}x)"
+    print(f"PARITY {name}: n={got.size} worst |x-y|/allowed = {worst:.3g}, "
+          f"bitwise different = {float((got != want).mean()):.3g}")    # shown with pytest -s
     return worst
 
 
@@ -76,8 +78,10 @@ def assert_bf16_close(name: str, got: np.ndarray, want: np.ndarray):
     ulp, frac = bf16_mismatch(got, want)
     assert ulp <= BF16_MAX_ULP, f"{name}: BF16 params up to {ulp} ulp apart"
     assert frac <= BF16_MAX_FRACTION, f"{name}: {frac:.3g} of BF16 params differ"
+    print(f"PARITY {name}: n={got.size} max ulp = {ulp}, fraction differing = {frac:.3g}")
     return ulp, frac
 
 
 def assert_norm_close(got: float, want: float):
     assert abs(got - want) <= NORM_RTOL * abs(want), f"norm {got!r} vs oracle {want!r}"
+    print(f"PARITY norm: {got!r} vs oracle {want!r}, relative error {abs(got - want) / abs(want):.3g}")

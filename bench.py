@@ -152,10 +152,10 @@ def layer_of_rank(rank: int) -> int:
 
 def max_over_ranks(x: float, world: int, device="cuda") -> float:
     """The slowest rank's time: multi-GPU numbers are device times, max over ranks."""
-    if world == 1:
+    import torch.distributed as dist
+    if world == 1 and not (dist.is_available() and dist.is_initialized()):
         return x
     import torch
-    import torch.distributed as dist
     t = torch.tensor([x], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
@@ -182,11 +182,14 @@ def run_cuda(args):
         raise SystemExit("bench.py needs a CUDA device: libslidedp has no CPU path "
                          "(use --impl reference for the CPU oracle)")
     torch.cuda.set_device(local)
-    if world > 1:
+    # under a launcher (torchrun sets RANK and MASTER_ADDR) the process group is used even for
+    # one rank, so that the N = 1 run exercises the same barrier / reduction code as N > 1
+    grouped = world > 1 or ("RANK" in os.environ and "MASTER_ADDR" in os.environ)
+    if grouped:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     def barrier():
-        if world > 1:
+        if grouped:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -321,7 +324,7 @@ def run_cuda(args):
             "clocks": clocks, "host_resident": host,
         }
     ctx.slidedp_destroy()
-    if world > 1:
+    if grouped:
         dist.barrier()
         dist.destroy_process_group()
     if out is not None:

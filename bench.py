@@ -321,7 +321,7 @@ def run_cuda(args):
                        "parallelism": f"{world} independent layer(s), one per GPU, no collective",
                        "l2": "inputs (8.1 GB touched per step) exceed the 126 MB L2"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
-            "clocks": clocks, "host_resident": host,
+            "clocks": clocks, "host_resident": host, "host_placement": host_placement(torch, local),
         }
     ctx.slidedp_destroy()
     if grouped:
@@ -540,6 +540,35 @@ def host_resident_report(ctx, sd, W, torch, dev):
                          for k in ("ms_norm", "ms_h2d", "ms_kernel", "ms_d2h")}}
 
 
+def host_placement(torch, local: int):
+    """Where the pinned state and the GPU sit (the paper keeps pinned buffers and the update
+    worker on a fixed NUMA node, Sec. 3.2 "Routes and physical resources"): NUMA nodes visible to
+    this process, the GPU's node as sysfs reports it, and the CPUs this process may run on."""
+    def read(path):
+        try:
+            with open(path) as f:
+                return f.read().strip()
+        except OSError:
+            return None
+    nodes = [d for d in os.listdir("/sys/devices/system/node")
+             if d.startswith("node") and d[4:].isdigit()] if os.path.isdir("/sys/devices/system/node") else []
+    bdf = None
+    try:
+        bdf = torch.cuda.get_device_properties(local).pci_bus_id
+        bdf = f"{torch.cuda.get_device_properties(local).pci_domain_id:04x}:{bdf:02x}:" \
+              f"{torch.cuda.get_device_properties(local).pci_device_id:02x}.0"
+    except Exception:
+        bdf = None
+    mems = None
+    status = read("/proc/self/status") or ""
+    for line in status.splitlines():
+        if line.startswith("Mems_allowed_list"):
+            mems = line.split(":", 1)[1].strip()
+    return {"numa_nodes": len(nodes), "mems_allowed": mems,
+            "gpu_numa_node": read(f"/sys/bus/pci/devices/{bdf}/numa_node") if bdf else None,
+            "cpus": len(os.sched_getaffinity(0))}
+
+
 def cpu_baseline(W, torch, np, wl, grads, layer):
     """The oracle as it stands, one whole step (norm + update) of the same layer on the host
     cores of this machine."""
@@ -555,9 +584,16 @@ def cpu_baseline(W, torch, np, wl, grads, layer):
     t0 = time.perf_counter()
     oracle.step(hg, w, m, v, p, oracle.HParams(step=2, **kw), nthreads=cores)
     dt = time.perf_counter() - t0
+    # the same oracle on ONE thread, on the first 2^24 parameters
+    k = min(n, 1 << 24)
+    t0 = time.perf_counter()
+    oracle.step([g[:k] for g in hg], w[:k], m[:k], v[:k], p[:k], oracle.HParams(step=3, **kw),
+                nthreads=1)
+    dt1 = time.perf_counter() - t0
     return {"value": n / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"one whole step (norm + update) over {n} of {wl.numel} parameters, R={wl.R}",
-            "seconds": dt}
+            "seconds": dt, "single_thread_value": k / dt1 / 1e9,
+            "single_thread_sample": f"one whole step over the first {k} parameters"}
 
 
 def main():

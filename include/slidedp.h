@@ -135,6 +135,9 @@ SLIDEDP_API int slidedp_grad_norm_finish(slidedp_ctx* ctx, double max_norm, doub
  * slidedp_grad_norm_finish must have been enqueued earlier on the same stream
  * (SLIDEDP_ERR_NO_NORM if none was ever issued on this context).
  * Asynchronous on cuda_stream; traffic is 26 + 2R bytes per parameter.
+ * master, m and v may also be PINNED HOST pointers (unified addressing): the kernel then reads and
+ * writes host memory directly, with no device slots at all. That needs no GPU memory budget but
+ * reaches less of the host link than slidedp_stream_step (measured 40 vs 47 GB/s each way).
  */
 SLIDEDP_API int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
                                float* master, float* m, float* v, void* param_bf16_out,

@@ -246,3 +246,25 @@ def test_async_layers_share_the_slot_ring_and_match_the_synchronous_step(ctx, sd
     ctx.slidedp_deliver_params(host[0], nl, out, 1 << 18, 2)
     assert np.array_equal(parity.u16(out), parity.u16(dp))
     ctx.slidedp_stream_wait()
+
+
+def test_zero_copy_update_on_pinned_host_state_matches_the_device_path(ctx, sd):
+    """With unified addressing the fused kernel can read and write pinned host state directly
+    (no slots at all): same bits as the device-resident update."""
+    n, R = (1 << 21) + 13, 4
+    g = torch.Generator(device="cuda").manual_seed(31)
+    dg = [(torch.randn(n, generator=g, device="cuda") * 1e-3).to(torch.bfloat16) for _ in range(R)]
+    w = torch.randn(n, generator=g, device="cuda") * 0.02
+    m = torch.randn(n, generator=g, device="cuda") * 3e-4
+    v = torch.randn(n, generator=g, device="cuda").square() * 1e-7
+    hw, hm, hv = pinned(parity.f32(w)), pinned(parity.f32(m)), pinned(parity.f32(v))
+    hp = sd.HParams(inv_R=0.25, max_norm=0.01, step=5)
+    ctx.slidedp_grad_norm(dg, n, 0.25, True)
+    ctx.slidedp_grad_norm_finish(0.01)
+    dp, zp = (torch.zeros(n, dtype=torch.bfloat16, device="cuda") for _ in range(2))
+    ctx.slidedp_reduce_adamw_chunk(dg, n, w, m, v, dp, hp)
+    ctx.slidedp_reduce_adamw_chunk(dg, n, hw, hm, hv, zp, hp)
+    torch.cuda.synchronize()
+    for a, b in ((hw, w), (hm, m), (hv, v)):
+        assert np.array_equal(a.numpy(), parity.f32(b))
+    assert np.array_equal(parity.u16(zp), parity.u16(dp))

@@ -1,0 +1,93 @@
+/* The C ABI used from plain C, with no Python in between: one clipped step of a small chunk
+ * through libslidedp, compared with the C oracle under the benchmark's tolerances. Built and
+ * run by tests/test_c_abi_program.py (gcc, links libslidedp, the oracle and the CUDA runtime).
+ * Exit code 0 and a line starting with "PASS" on success. */
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "slidedp.h"
+#include "slidedp_oracle.h"
+
+#define CHECK_CUDA(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) { \
+  printf("FAIL cuda %s at line %d\n", cudaGetErrorString(e_), __LINE__); return 2; } } while (0)
+#define CHECK_SD(x) do { int r_ = (x); if (r_ != SLIDEDP_OK) { \
+  printf("FAIL libslidedp: %s at line %d\n", slidedp_strerror(r_), __LINE__); return 3; } } while (0)
+
+static uint32_t lcg(uint32_t* s) { *s = *s * 1664525u + 1013904223u; return *s; }
+static float uniform(uint32_t* s) { return (float)(lcg(s) >> 8) / 16777216.0f - 0.5f; }
+
+int main(void) {
+  enum { R = 3 };
+  const int64_t n = 100003;
+  uint32_t seed = 12345u;
+  uint16_t* hg[R];
+  float *hw = malloc(n * 4), *hm = malloc(n * 4), *hv = malloc(n * 4);
+  uint16_t* hp = malloc(n * 2);
+  for (int r = 0; r < R; ++r) {
+    hg[r] = malloc(n * 2);
+    for (int64_t i = 0; i < n; ++i) hg[r][i] = oracle_f32_to_bf16(4e-3f * uniform(&seed));
+  }
+  for (int64_t i = 0; i < n; ++i) {
+    hw[i] = 0.05f * uniform(&seed);
+    hm[i] = 1e-3f * uniform(&seed);
+    hv[i] = 1e-6f * (uniform(&seed) + 0.5f);
+  }
+  slidedp_hparams hp_sd = {1e-5, 0.9, 0.95, 1e-8, 0.1, 1.0 / R, 0.05, 7};
+  oracle_hparams hp_or = {1e-5, 0.9, 0.95, 1e-8, 0.1, 1.0 / R, 0.05, 7};
+
+  /* device side */
+  void* dg[R];
+  float *dw, *dm, *dv;
+  void* dp;
+  for (int r = 0; r < R; ++r) {
+    CHECK_CUDA(cudaMalloc(&dg[r], n * 2));
+    CHECK_CUDA(cudaMemcpy(dg[r], hg[r], n * 2, cudaMemcpyHostToDevice));
+  }
+  CHECK_CUDA(cudaMalloc((void**)&dw, n * 4)); CHECK_CUDA(cudaMalloc((void**)&dm, n * 4));
+  CHECK_CUDA(cudaMalloc((void**)&dv, n * 4)); CHECK_CUDA(cudaMalloc(&dp, n * 2));
+  CHECK_CUDA(cudaMemcpy(dw, hw, n * 4, cudaMemcpyHostToDevice));
+  CHECK_CUDA(cudaMemcpy(dm, hm, n * 4, cudaMemcpyHostToDevice));
+  CHECK_CUDA(cudaMemcpy(dv, hv, n * 4, cudaMemcpyHostToDevice));
+  slidedp_ctx* ctx = NULL;
+  CHECK_SD(slidedp_create(&ctx, 0, 0));
+  double norm = 0, coef = 0;
+  CHECK_SD(slidedp_grad_norm(ctx, (const void* const*)dg, R, n, 1.0 / R, 1, NULL));
+  CHECK_SD(slidedp_grad_norm_finish(ctx, hp_sd.max_norm, &norm, &coef, NULL));
+  CHECK_SD(slidedp_reduce_adamw_chunk(ctx, (const void* const*)dg, R, n, dw, dm, dv, dp, &hp_sd, NULL));
+  CHECK_CUDA(cudaDeviceSynchronize());
+  float *gw = malloc(n * 4), *gm = malloc(n * 4), *gv = malloc(n * 4);
+  uint16_t* gp = malloc(n * 2);
+  CHECK_CUDA(cudaMemcpy(gw, dw, n * 4, cudaMemcpyDeviceToHost));
+  CHECK_CUDA(cudaMemcpy(gm, dm, n * 4, cudaMemcpyDeviceToHost));
+  CHECK_CUDA(cudaMemcpy(gv, dv, n * 4, cudaMemcpyDeviceToHost));
+  CHECK_CUDA(cudaMemcpy(gp, dp, n * 2, cudaMemcpyDeviceToHost));
+  const int64_t launches = slidedp_kernel_launches(ctx);
+  CHECK_SD(slidedp_destroy(ctx));
+
+  /* oracle side */
+  double onorm = 0, ocoef = 0;
+  if (oracle_step((const uint16_t* const*)hg, R, n, hw, hm, hv, hp, 0, &hp_or, &onorm, &ocoef, 1)) {
+    printf("FAIL oracle_step\n");
+    return 4;
+  }
+  int64_t bad = 0, bf16_differ = 0;
+  const float* got[3] = {gw, gm, gv};
+  const float* want[3] = {hw, hm, hv};
+  for (int a = 0; a < 3; ++a)
+    for (int64_t i = 0; i < n; ++i) {
+      const double y = want[a][i], err = fabs((double)got[a][i] - y);
+      const double allowed = fmax(1e-6 * fabs(y), 1e-12);
+      if (!(err <= allowed)) ++bad;
+    }
+  for (int64_t i = 0; i < n; ++i) bf16_differ += gp[i] != hp[i];
+  const int ok = bad == 0 && bf16_differ <= n / 10000 && fabs(norm - onorm) <= 1e-6 * onorm &&
+                 fabs(coef - ocoef) <= 1e-6 * ocoef && ocoef < 1.0 && launches == 3;
+  printf("%s n=%lld R=%d norm=%.12g (oracle %.12g) coef=%.6f fp32_outside=%lld bf16_differ=%lld launches=%lld\n",
+         ok ? "PASS" : "FAIL", (long long)n, R, norm, onorm, coef, (long long)bad,
+         (long long)bf16_differ, (long long)launches);
+  return ok ? 0 : 1;
+}

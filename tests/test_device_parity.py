@@ -344,3 +344,52 @@ def test_guard_bands_around_every_buffer_stay_intact(ctx, sd, n):
     ctx.slidedp_deliver_params(host, n, p, 8, 2)
     assert torch.all(pfull[:pad] == -7.0) and torch.all(pfull[pad + n:] == -7.0)
     assert torch.equal(p, w.to(torch.bfloat16))
+
+
+def test_random_hyperparameters_and_steps(ctx, sd):
+    """Forty seeded draws of (lr, betas, eps, weight decay, step, clip, R) on a ragged chunk."""
+    rng = np.random.default_rng(2024)
+    n = 4099
+    for case in range(40):
+        R = int(rng.integers(1, 17))
+        kw = dict(lr=float(10 ** rng.uniform(-6, -2)), beta1=float(rng.choice([0.0, 0.5, 0.8, 0.9, 0.99])),
+                  beta2=float(rng.choice([0.0, 0.9, 0.95, 0.999, 0.9999])),
+                  eps=float(10 ** rng.uniform(-12, -5)), weight_decay=float(rng.choice([0.0, 0.01, 0.1, 1.0])),
+                  step=int(rng.choice([1, 2, 10, 1000, 10 ** 6])))
+        clip = float(rng.choice([0.0, 1e-3, 1.0, 1e3]))
+        grads, w, m, v = random_case(n, R, seed=5000 + case, zero_moments=bool(case % 3 == 0),
+                                     sigma=float(10 ** rng.uniform(-5, -1)))
+        got, want = run_both(ctx, sd, grads, w, m, v, kw, clip)
+        assert_parity(f"case {case}: R={R} clip={clip} {kw}", got, want, clip)
+
+
+def test_whole_step_replays_from_a_cuda_graph(ctx, sd):
+    """Norm, finish and update only enqueue work on the caller's stream (no allocation, no
+    synchronisation), so a step can be captured once and replayed; the replay gives the bits of
+    the eager step."""
+    n, R = (1 << 18) + 5, 4
+    grads, w, m, v = random_case(n, R, seed=42)
+    dg = [g.cuda() for g in grads]
+    hp = sd.HParams(inv_R=0.25, max_norm=0.02, step=2)
+
+    def fresh():
+        return w.cuda(), m.cuda(), v.cuda(), torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+
+    def step(state):
+        ctx.slidedp_grad_norm(dg, n, 0.25, True)
+        ctx.slidedp_grad_norm_finish(0.02)
+        ctx.slidedp_reduce_adamw_chunk(dg, n, *state, hp)
+
+    eager = fresh()
+    step(eager)
+    torch.cuda.synchronize()
+    replayed = fresh()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step(replayed)
+    for t, src in zip(replayed, fresh()):
+        t.copy_(src)                      # capture does not execute: start from the same state
+    graph.replay()
+    torch.cuda.synchronize()
+    for a, b in zip(eager, replayed):
+        assert torch.equal(a, b)

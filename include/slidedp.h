@@ -143,6 +143,20 @@ SLIDEDP_API int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* 
                                float* master, float* m, float* v, void* param_bf16_out,
                                const slidedp_hparams* hp, void* cuda_stream);
 
+/* ---- rank reduction alone ---------------------------------------------------------------------
+ *
+ * The paper's GPU-reduction route (Sec. 3.2 "Gradient return"): the rank-local gradients are summed,
+ * averaged, and ONE gradient of the layer's size is returned for the copy to the host, where the
+ * paper's CPU update consumes it. For callers that keep that route:
+ *   out_bf16[i] = bf16_rne( fl32( ((g_0[i] + g_1[i]) + ... + g_{R-1}[i]) in FP32 ) * (float)inv_R )
+ * (the fused update above does NOT round the average to BF16; this entry point exists for the
+ * paper's data path, not for slidedp_reduce_adamw_chunk). grads_bf16: host array of R device
+ * pointers; out_bf16: device, n BF16 values, 16-byte aligned, may not overlap the inputs.
+ * Asynchronous on cuda_stream; traffic 2R + 2 bytes per parameter.
+ */
+SLIDEDP_API int slidedp_reduce_mean_bf16(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                             double inv_R, void* out_bf16, void* cuda_stream);
+
 /* ---- host-resident update: state in pinned host memory, streamed chunk by chunk -------
  *
  * host_master / host_m / host_v: PINNED host arrays of n_total floats, updated in place.

@@ -76,6 +76,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_reduce_mean.restype = None
         L.oracle_reduce_mean.argtypes = [pp, ctypes.c_int, ctypes.c_int64, ctypes.c_double,
                                          ctypes.c_void_p]
+        L.oracle_reduce_mean_bf16.restype = None
+        L.oracle_reduce_mean_bf16.argtypes = [pp, ctypes.c_int, ctypes.c_int64, ctypes.c_double,
+                                              ctypes.c_void_p]
         L.oracle_grad_sumsq.restype = ctypes.c_double
         L.oracle_grad_sumsq.argtypes = [pp, ctypes.c_int, ctypes.c_int64, ctypes.c_double,
                                         ctypes.c_int]
@@ -140,6 +143,13 @@ def reduce_mean(grads, inv_R: float) -> np.ndarray:
     ptrs, R, n = _grad_ptrs(grads)
     out = np.empty(n, np.float32)
     lib().oracle_reduce_mean(ptrs, R, n, inv_R, out.ctypes.data)
+    return out
+
+
+def reduce_mean_bf16(grads, inv_R: float) -> np.ndarray:
+    ptrs, R, n = _grad_ptrs(grads)
+    out = np.empty(n, np.uint16)
+    lib().oracle_reduce_mean_bf16(ptrs, R, n, inv_R, out.ctypes.data)
     return out
 
 

@@ -59,6 +59,12 @@ void oracle_reduce_mean(const uint16_t* const* grads, int R, int64_t n, double i
   for (int64_t i = 0; i < n; ++i) gbar[i] = mean_of_ranks(grads, R, i, inv_R32);
 }
 
+void oracle_reduce_mean_bf16(const uint16_t* const* grads, int R, int64_t n, double inv_R,
+                             uint16_t* out) {
+  const float inv_R32 = (float)inv_R;
+  for (int64_t i = 0; i < n; ++i) out[i] = oracle_f32_to_bf16(mean_of_ranks(grads, R, i, inv_R32));
+}
+
 /* ---- global L2 norm of the averaged gradient (not in the paper) ----------- */
 double oracle_grad_sumsq(const uint16_t* const* grads, int R, int64_t n, double inv_R,
                          int nthreads) {

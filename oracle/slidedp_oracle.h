@@ -64,6 +64,11 @@ uint16_t oracle_f32_to_bf16(float x);
 void oracle_reduce_mean(const uint16_t* const* grads, int R, int64_t n, double inv_R,
                         float* gbar);
 
+/* The paper's GPU-reduction route returns ONE BF16 gradient per layer to the host (Sec. 3.2
+ * "Gradient return"): out[i] = round-to-nearest-even BF16 of gbar[i] as defined above. */
+void oracle_reduce_mean_bf16(const uint16_t* const* grads, int R, int64_t n, double inv_R,
+                             uint16_t* out);
+
 /* Sum over i of double(gbar[i])^2 for the averaged gradient of one chunk. */
 double oracle_grad_sumsq(const uint16_t* const* grads, int R, int64_t n, double inv_R,
                          int nthreads);

@@ -289,4 +289,49 @@ cast_master_to_bf16_kernel(const float* __restrict__ master, int64_t n,
   }
 }
 
+// ---- rank reduction alone: the averaged gradient as one BF16 buffer --------------------
+//
+// The paper's GPU-reduction route materialises ONE gradient of G_l bytes per layer for the copy
+// to the host (Sec. 3.2 "Gradient return"). Same left-to-right FP32 sum and FP32 multiply by
+// (float)1/R as the fused kernel, then one round-to-nearest-even to BF16. Eight elements per
+// thread; 2R + 2 bytes of traffic per parameter.
+constexpr int kReduceThreads = 256;
+template <int R>
+__global__ void __launch_bounds__(kReduceThreads)
+reduce_mean_bf16_kernel(GradPtrs gp, int64_t n, float inv_R, uint16_t* __restrict__ out) {
+  const int64_t base = ((int64_t)blockIdx.x * kReduceThreads + threadIdx.x) * 8;
+  if (base >= n) return;
+  if (base + 8 <= n) {
+    uint4 graw[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) graw[r] = ld_stream(gp.p[r] + base);
+    float s[8];
+    {
+      const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[0]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { s[2 * j] = bf16_lo(x[j]); s[2 * j + 1] = bf16_hi(x[j]); }
+    }
+#pragma unroll
+    for (int r = 1; r < R; ++r) {
+      const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[r]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        s[2 * j] = __fadd_rn(s[2 * j], bf16_lo(x[j]));
+        s[2 * j + 1] = __fadd_rn(s[2 * j + 1], bf16_hi(x[j]));
+      }
+    }
+    uint32_t b[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) b[j] = f32_to_bf16_bits(__fmul_rn(s[j], inv_R));
+    st_stream(out + base, make_uint4(b[0] | (b[1] << 16), b[2] | (b[3] << 16),
+                                     b[4] | (b[5] << 16), b[6] | (b[7] << 16)));
+  } else {
+    for (int64_t i = base; i < n; ++i) {
+      float t = __uint_as_float((uint32_t)gp.p[0][i] << 16);
+      for (int r = 1; r < R; ++r) t = __fadd_rn(t, __uint_as_float((uint32_t)gp.p[r][i] << 16));
+      out[i] = (uint16_t)f32_to_bf16_bits(__fmul_rn(t, inv_R));
+    }
+  }
+}
+
 }  // namespace slidedp

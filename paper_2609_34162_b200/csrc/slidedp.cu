@@ -564,6 +564,35 @@ int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* grads_bf16, 
                        static_cast<cudaStream_t>(cuda_stream));
 }
 
+int slidedp_reduce_mean_bf16(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                             double inv_R, void* out_bf16, void* cuda_stream) {
+  if (!ctx || n < 0 || inv_R != inv_R) return SLIDEDP_ERR_INVALID_ARG;
+  GradPtrs gp;
+  int rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  if (n > 0 && !out_bf16) return SLIDEDP_ERR_INVALID_ARG;
+  if (!aligned16(out_bf16)) return SLIDEDP_ERR_MISALIGNED;
+  if (n == 0) return SLIDEDP_OK;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const unsigned blocks = (unsigned)((n + 8 * kReduceThreads - 1) / (8 * kReduceThreads));
+  uint16_t* out = static_cast<uint16_t*>(out_bf16);
+  const float inv = (float)inv_R;
+  switch (R) {
+#define SLIDEDP_CASE(r) \
+  case r: reduce_mean_bf16_kernel<r><<<blocks, kReduceThreads, 0, st>>>(gp, n, inv, out); break;
+    SLIDEDP_CASE(1) SLIDEDP_CASE(2) SLIDEDP_CASE(3) SLIDEDP_CASE(4) SLIDEDP_CASE(5) SLIDEDP_CASE(6)
+    SLIDEDP_CASE(7) SLIDEDP_CASE(8) SLIDEDP_CASE(9) SLIDEDP_CASE(10) SLIDEDP_CASE(11)
+    SLIDEDP_CASE(12) SLIDEDP_CASE(13) SLIDEDP_CASE(14) SLIDEDP_CASE(15) SLIDEDP_CASE(16)
+#undef SLIDEDP_CASE
+    default: return SLIDEDP_ERR_INVALID_ARG;
+  }
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  return SLIDEDP_OK;
+}
+
 int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n_total,
                         float* host_master, float* host_m, float* host_v, void* param_bf16_out,
                         int64_t chunk_elems, int nbuf, int norm_ready,

@@ -86,6 +86,8 @@ _lib.slidedp_stream_step.restype = ctypes.c_int
 _lib.slidedp_stream_step.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp, _vp,
                                      ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                      ctypes.POINTER(_HParams), ctypes.POINTER(_Stats)]
+_lib.slidedp_reduce_mean_bf16.restype = ctypes.c_int
+_lib.slidedp_reduce_mean_bf16.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, ctypes.c_double, _vp, _vp]
 _lib.slidedp_stream_step_async.restype = ctypes.c_int
 _lib.slidedp_stream_step_async.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp, _vp,
                                            ctypes.c_int64, ctypes.c_int, ctypes.c_int,
@@ -217,6 +219,10 @@ class Context:
         self._check(_lib.slidedp_reduce_adamw_chunk(
             self._h, _grad_array(grads), len(grads), n, _ptr(master), _ptr(m), _ptr(v),
             _ptr(param_bf16_out), ctypes.byref(c), _stream(stream)))
+
+    def slidedp_reduce_mean_bf16(self, grads, n: int, inv_R: float, out_bf16, stream=None) -> None:
+        self._check(_lib.slidedp_reduce_mean_bf16(self._h, _grad_array(grads), len(grads), n, inv_R,
+                                                  _ptr(out_bf16), _stream(stream)))
 
     def slidedp_stream_step(self, grads, n_total: int, host_master, host_m, host_v,
                             param_bf16_out, chunk_elems: int, nbuf: int, hp: HParams,

@@ -393,3 +393,19 @@ def test_whole_step_replays_from_a_cuda_graph(ctx, sd):
     torch.cuda.synchronize()
     for a, b in zip(eager, replayed):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("R", [1, 2, 3, 4, 7, 8, 16])
+def test_rank_reduction_alone_returns_the_bf16_mean_bit_exact(ctx, sd, R):
+    for n in (0, 5, 8, 4099, (1 << 20) + 7):
+        g = torch.Generator().manual_seed(100 * R + n % 89)
+        scale = 2.0 ** torch.randint(-10, 1, (R, max(n, 1)), generator=g).float()
+        grads = [(torch.randn(max(n, 1), generator=g) * 1e-2 * scale[r]).to(torch.bfloat16)[:n]
+                 for r in range(R)]
+        out = torch.full((max(n, 8),), 9.0, dtype=torch.bfloat16, device="cuda")
+        dg = [x.cuda() for x in grads] if n else [out] * R      # n = 0 still needs real pointers
+        ctx.slidedp_reduce_mean_bf16(dg, n, 1.0 / R, out)
+        torch.cuda.synchronize()
+        want = oracle.reduce_mean_bf16([parity.u16(x) for x in grads], 1.0 / R) if n else np.zeros(0, np.uint16)
+        assert np.array_equal(parity.u16(out[:n]), want), (R, n)
+        assert torch.all(out[n:] == 9.0)

@@ -430,3 +430,19 @@ def test_delivery_cast_matches_torch_cast_and_keeps_specials():
     nan = oracle.cast_master_to_bf16(np.array([np.nan], np.float32))[0]
     assert (nan & 0x7F80) == 0x7F80 and (nan & 0x7F) != 0
     assert oracle.cast_master_to_bf16(np.zeros(0, np.float32)).size == 0
+
+
+# ------------------------------------------------ rank reduction returned as one BF16 gradient
+@pytest.mark.parametrize("R", [1, 2, 3, 8])
+def test_reduced_bf16_gradient_is_the_cast_of_the_fp32_mean(R):
+    rng = np.random.default_rng(16 + R)
+    n = 5000
+    grads = [rand_bf16(rng, n, 2e-3) for _ in range(R)]
+    got = oracle.reduce_mean_bf16(grads, 1.0 / R)
+    assert np.array_equal(got, bf16_bits(oracle.reduce_mean(grads, 1.0 / R)))   # torch's cast
+    if R in (1, 2, 8):       # identical ranks and a power-of-two R: the gradient itself comes back
+        same = oracle.reduce_mean_bf16([grads[0]] * R, 1.0 / R)
+        assert np.array_equal(same, grads[0])
+    # hand case: (1 + 2^-7) averaged with 1 is 1 + 2^-8, a BF16 tie that rounds to the even 1.0
+    a = bf16_bits(np.array([1.0078125], np.float32)); b = bf16_bits(np.array([1.0], np.float32))
+    assert oracle.reduce_mean_bf16([a, b], 0.5)[0] == 0x3F80

@@ -25,7 +25,7 @@
  *   clipping   not in the paper: global L2 norm of the averaged gradient over
  *              all parameters of the step, coefficient min(1, max/(norm+1e-6)).
  *              The 1e-6 constant and the left-to-right rank order are
- *              definitions fixed by this build (parity unpinned by the paper);
+ *              definitions fixed by this library (parity unpinned by the paper);
  *              everything else is pinned by the CPU tests.
  *
  * All pointers are host pointers. BF16 values travel as uint16_t bit patterns.

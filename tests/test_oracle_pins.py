@@ -446,3 +446,60 @@ def test_reduced_bf16_gradient_is_the_cast_of_the_fp32_mean(R):
     # hand case: (1 + 2^-7) averaged with 1 is 1 + 2^-8, a BF16 tie that rounds to the even 1.0
     a = bf16_bits(np.array([1.0078125], np.float32)); b = bf16_bits(np.array([1.0], np.float32))
     assert oracle.reduce_mean_bf16([a, b], 0.5)[0] == 0x3F80
+
+
+# ------------------------------------------------------------ invariants of Adam and of clipping
+def test_adam_is_invariant_to_the_gradient_scale_when_eps_is_zero():
+    """From zero moments with eps = 0, multiplying every gradient by a power of two scales m by
+    it and v by its square exactly, so mhat / sqrt(vhat), and with it the master, must come out
+    bit-identical at every step (Kingma & Ba Sec. 2.1: the step is invariant to gradient scale)."""
+    rng = np.random.default_rng(17)
+    n, R, T = 3000, 1, 5            # one rank: the mean cannot cancel to zero (0/0 with eps = 0)
+    a = fresh_state(rng, n, zero_moments=True); b = tuple(x.copy() for x in a)
+    pa, pb = np.zeros(n, np.uint16), np.zeros(n, np.uint16)
+    for t in range(1, T + 1):
+        grads = [rand_bf16(rng, n, 1e-3) for _ in range(R)]
+        scaled = [bf16_bits(bf16_values(g) * np.float32(64.0)) for g in grads]
+        hp = HParams(lr=1e-4, beta1=0.9, beta2=0.95, eps=0.0, weight_decay=0.1, inv_R=1.0, step=t)
+        # gradients that are exactly zero would give 0/0 with eps = 0: nudge them
+        for g, s in zip(grads, scaled):
+            z = (g & 0x7FFF) == 0
+            g[z] = 0x3A80; s[z] = bf16_bits(bf16_values(g[z]) * np.float32(64.0))
+        oracle.reduce_adamw_chunk(grads, *a, pa, hp)
+        oracle.reduce_adamw_chunk(scaled, *b, pb, hp)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(pa, pb)
+        assert np.array_equal(b[1], a[1] * np.float32(64.0))
+        assert np.array_equal(b[2], a[2] * np.float32(4096.0))
+
+
+def test_active_clipping_cancels_a_common_gradient_scale():
+    """While the norm exceeds max_norm the clipped gradient is g * max_norm / (norm + 1e-6):
+    doubling every gradient doubles the norm exactly, so the clipped gradient changes only
+    through the 1e-6 in the denominator."""
+    rng = np.random.default_rng(18)
+    n, R = 8000, 4
+    grads = [rand_bf16(rng, n, 5e-2) for _ in range(R)]
+    doubled = [bf16_bits(bf16_values(g) * np.float32(2.0)) for g in grads]
+    a = fresh_state(rng, n); b = tuple(x.copy() for x in a)
+    pa, pb = np.zeros(n, np.uint16), np.zeros(n, np.uint16)
+    hp = HParams(inv_R=0.25, max_norm=1.0, step=4)
+    na, ca = oracle.step(grads, *a, pa, hp)
+    nb, cb = oracle.step(doubled, *b, pb, hp)
+    assert na > 1.0 and nb == 2.0 * na
+    assert abs(2.0 * cb / ca - 1.0) < 1e-6            # 2 c' = c (1 + O(1e-6 / norm))
+    for x, y in zip(a, b):      # equal up to that 1e-6 (absolute scale: m can cancel to near 0)
+        assert np.allclose(x, y, rtol=2e-6, atol=2e-6 * float(np.abs(x).max()))
+    assert not all(np.array_equal(x, y) for x, y in zip(a, b))     # and the 1e-6 is really there
+
+
+@pytest.mark.parametrize("R", [3, 4, 8])
+def test_permuting_the_ranks_moves_the_fp32_sum_by_rounding_only(R):
+    rng = np.random.default_rng(19 + R)
+    n = 4096
+    grads = [rand_bf16(rng, n, 1e-3 * 2.0 ** (-9 * (r % 3))) for r in range(R)]  # spread exponents
+    base = oracle.reduce_mean(grads, 1.0 / R)
+    perm = oracle.reduce_mean(grads[::-1], 1.0 / R)
+    exact = sum(bf16_values(g).astype(np.float64) for g in grads) / R
+    assert ulp_diff(base, perm).max() <= R                       # a few ulps at most ...
+    assert np.allclose(base, exact, rtol=R * 6e-8, atol=1e-12)   # ... around the exact mean
+    assert (base != perm).any() or R < 3

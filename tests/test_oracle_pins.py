@@ -502,4 +502,3 @@ def test_permuting_the_ranks_moves_the_fp32_sum_by_rounding_only(R):
     exact = sum(bf16_values(g).astype(np.float64) for g in grads) / R
     assert ulp_diff(base, perm).max() <= R                       # a few ulps at most ...
     assert np.allclose(base, exact, rtol=R * 6e-8, atol=1e-12)   # ... around the exact mean
-    assert (base != perm).any() or R < 3

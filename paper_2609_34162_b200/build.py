@@ -12,8 +12,11 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libslidedp.so")
-SOURCES = [os.path.join(CSRC, "slidedp.cu")]
-DEPENDS = SOURCES + [os.path.join(CSRC, "kernels.cuh"), os.path.join(ROOT, "include", "slidedp.h")]
+SOURCES = [os.path.join(CSRC, f) for f in ("common.cu", "context.cu", "update.cu", "stream.cu",
+                                           "model.cu")]
+DEPENDS = SOURCES + [os.path.join(CSRC, f) for f in ("kernels.cuh", "cast_kernel.cuh",
+                                                     "device_utils.cuh", "types.h", "internal.h")]
+DEPENDS.append(os.path.join(ROOT, "include", "slidedp.h"))
 
 
 def nvcc() -> str:

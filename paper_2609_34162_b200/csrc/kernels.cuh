@@ -9,9 +9,11 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "device_utils.cuh"
+#include "types.h"
+
 namespace slidedp {
 
-constexpr int kMaxRanks = 16;
 constexpr int kVec = 4;                 // parameters per thread in the update kernel
 constexpr int kUpdateThreads = 128;
 constexpr int kNormVec = 8;             // elements per thread per load in the norm kernel
@@ -19,43 +21,6 @@ constexpr int kNormThreads = 256;
 constexpr int kNormIters = 8;
 constexpr int kNormTile = kNormThreads * kNormVec * kNormIters;   // 16384 elements per partial
 constexpr int kFinishThreads = 1024;
-
-struct GradPtrs {
-  const uint16_t* p[kMaxRanks];
-};
-
-// Everything the update needs that does not depend on the element, prepared on the host
-// in double from the double-typed hyper-parameters.
-struct UpdateConsts {
-  double beta1, beta2;
-  double omb1, omb2;        // 1 - beta1, 1 - beta2 (exact in double for beta in [0.5, 1))
-  double rsqrt_bc2;         // 1 / sqrt(1 - beta2^t)
-  double eps;
-  double neg_lr_over_bc1;   // -lr / (1 - beta1^t)
-  double decay;             // 1 - lr * weight_decay
-  float inv_R;              // (float)inv_R
-};
-
-// ---- small helpers -----------------------------------------------------------------
-
-__device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xFFFF0000u); }
-
-// FP32 -> BF16 bits, round to nearest even, NaN stays NaN.
-__device__ __forceinline__ uint32_t f32_to_bf16_bits(float x) {
-  uint16_t r;
-  asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(x));
-  return (uint32_t)r;
-}
-
-// Streaming (read-once / write-once) 128-bit accesses: keep them out of L1 and mark them
-// evict-first in L2, since nothing on this path is ever re-read.
-__device__ __forceinline__ uint4 ld_stream(const void* p) {
-  return __ldcs(reinterpret_cast<const uint4*>(p));
-}
-__device__ __forceinline__ void st_stream(void* p, uint4 v) {
-  __stcs(reinterpret_cast<uint4*>(p), v);
-}
 
 // Hardware seeds for FP64 reciprocal square root and reciprocal (about 20 good bits; the
 // full double exponent range). One Newton step each below brings them to ~1e-12.
@@ -262,30 +227,6 @@ grad_norm_finish_kernel(const double* __restrict__ partials, int64_t count, doub
     scalars[1] = norm;
     scalars[2] = c;
     scalars[3] = (norm - norm == 0.0) ? 0.0 : 1.0;
-  }
-}
-
-// ---- parameter delivery: FP32 master -> BF16 copy --------------------------------------
-//
-// Eight elements per thread: two 16-byte loads, one 16-byte store, round to nearest even.
-// HBM traffic is 6 bytes per parameter, but the kernel always runs behind an H2D copy of the
-// same chunk (4 bytes per parameter over the host link), which is the bound.
-constexpr int kCastThreads = 256;
-__global__ void __launch_bounds__(kCastThreads)
-cast_master_to_bf16_kernel(const float* __restrict__ master, int64_t n,
-                           uint16_t* __restrict__ param_out) {
-  const int64_t base = ((int64_t)blockIdx.x * kCastThreads + threadIdx.x) * 8;
-  if (base >= n) return;
-  if (base + 8 <= n) {
-    const uint4 a = ld_stream(master + base), b = ld_stream(master + base + 4);
-    uint4 o;
-    o.x = f32_to_bf16_bits(__uint_as_float(a.x)) | (f32_to_bf16_bits(__uint_as_float(a.y)) << 16);
-    o.y = f32_to_bf16_bits(__uint_as_float(a.z)) | (f32_to_bf16_bits(__uint_as_float(a.w)) << 16);
-    o.z = f32_to_bf16_bits(__uint_as_float(b.x)) | (f32_to_bf16_bits(__uint_as_float(b.y)) << 16);
-    o.w = f32_to_bf16_bits(__uint_as_float(b.z)) | (f32_to_bf16_bits(__uint_as_float(b.w)) << 16);
-    st_stream(param_out + base, o);
-  } else {
-    for (int64_t i = base; i < n; ++i) param_out[i] = (uint16_t)f32_to_bf16_bits(master[i]);
   }
 }
 

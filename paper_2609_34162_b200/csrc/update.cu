@@ -1,0 +1,243 @@
+// libslidedp: the device-resident path: kernel launchers, the global norm, the fused update, the
+// rank reduction alone and the norm variant that allocates nothing.
+// See include/slidedp.h for the contract of every entry point.
+#include "internal.h"
+#include "kernels.cuh"
+
+using namespace slidedp;
+using namespace slidedp::host;
+
+namespace slidedp {
+namespace host {
+
+template <int R_T>
+static void launch_update_t(const GradPtrs& gp, int /*R*/, int64_t n, float* w, float* m, float* v,
+                     uint16_t* p, const UpdateConsts& k, const double* coef, cudaStream_t st) {
+  const int64_t groups = (n + kVec - 1) / kVec;
+  const unsigned blocks = (unsigned)((groups + kUpdateThreads - 1) / kUpdateThreads);
+  reduce_adamw_kernel<R_T><<<blocks, kUpdateThreads, 0, st>>>(gp, n, w, m, v, p, k, coef);
+}
+
+int launch_update(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, float* w, float* m,
+                  float* v, uint16_t* p, const UpdateConsts& k, const double* coef,
+                  cudaStream_t st) {
+  if (n == 0) return SLIDEDP_OK;
+  // one instantiation per rank count: the R loads are fully unrolled (a runtime-R loop over a
+  // 16-entry register array ran at 4.0 TB/s for R = 3 against 6.4+ TB/s unrolled)
+  switch (R) {
+#define SLIDEDP_CASE(r) case r: launch_update_t<r>(gp, R, n, w, m, v, p, k, coef, st); break;
+    SLIDEDP_CASE(1) SLIDEDP_CASE(2) SLIDEDP_CASE(3) SLIDEDP_CASE(4) SLIDEDP_CASE(5) SLIDEDP_CASE(6)
+    SLIDEDP_CASE(7) SLIDEDP_CASE(8) SLIDEDP_CASE(9) SLIDEDP_CASE(10) SLIDEDP_CASE(11)
+    SLIDEDP_CASE(12) SLIDEDP_CASE(13) SLIDEDP_CASE(14) SLIDEDP_CASE(15) SLIDEDP_CASE(16)
+#undef SLIDEDP_CASE
+    default: return SLIDEDP_ERR_INVALID_ARG;
+  }
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  return SLIDEDP_OK;
+}
+
+// One instantiation per rank count (R is validated to 1..16 before this is reached).
+void launch_sumsq(const GradPtrs& gp, int R, int64_t n, float inv_R, double* tile_sums,
+                  unsigned blocks, cudaStream_t st) {
+  switch (R) {
+#define SLIDEDP_CASE(r) \
+  case r: grad_sumsq_tiles_kernel<r><<<blocks, kNormThreads, 0, st>>>(gp, n, inv_R, tile_sums); break;
+    SLIDEDP_CASE(1) SLIDEDP_CASE(2) SLIDEDP_CASE(3) SLIDEDP_CASE(4) SLIDEDP_CASE(5) SLIDEDP_CASE(6)
+    SLIDEDP_CASE(7) SLIDEDP_CASE(8) SLIDEDP_CASE(9) SLIDEDP_CASE(10) SLIDEDP_CASE(11)
+    SLIDEDP_CASE(12) SLIDEDP_CASE(13) SLIDEDP_CASE(14) SLIDEDP_CASE(15) SLIDEDP_CASE(16)
+#undef SLIDEDP_CASE
+    default: break;
+  }
+}
+
+static int ensure_partials(slidedp_ctx* ctx, int64_t need, cudaStream_t st) {
+  if (need <= ctx->partials_cap) return SLIDEDP_OK;
+  // Rare: a step of more than 17 G parameters. Growing keeps the tiles already written.
+  int64_t cap = ctx->partials_cap;
+  while (cap < need) cap *= 2;
+  double* bigger = nullptr;
+  CU(cudaMalloc(&bigger, (size_t)cap * sizeof(double)));
+  cudaError_t e = cudaMemcpyAsync(bigger, ctx->partials, (size_t)ctx->partials_used * sizeof(double),
+                                  cudaMemcpyDeviceToDevice, st);
+  if (e == cudaSuccess) {
+    int rc = bounded_stream_wait(ctx, st, kWaitSeconds);
+    if (rc != SLIDEDP_OK) { cudaFree(bigger); return rc; }
+  } else {
+    cudaFree(bigger);
+    return cuda_fail(ctx, e);
+  }
+  cudaFree(ctx->partials);
+  ctx->partials = bigger;
+  ctx->partials_cap = cap;
+  return SLIDEDP_OK;
+}
+
+int norm_chunk(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, double inv_R,
+               int first_chunk, cudaStream_t st) {
+  if (first_chunk) ctx->partials_used = 0;
+  if (n == 0) return SLIDEDP_OK;
+  const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
+  int rc = ensure_partials(ctx, ctx->partials_used + ntiles, st);
+  if (rc != SLIDEDP_OK) return rc;
+  // one block per tile: the hardware scheduler balances them, a tail of one tile at most
+  const unsigned blocks = (unsigned)ntiles;
+  double* dst = ctx->partials + ctx->partials_used;
+  const float inv = (float)inv_R;
+  launch_sumsq(gp, R, n, inv, dst, blocks, st);
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  ctx->partials_used += ntiles;
+  return SLIDEDP_OK;
+}
+
+int norm_finish(slidedp_ctx* ctx, double max_norm, cudaStream_t st) {
+  grad_norm_finish_kernel<<<1, kFinishThreads, 0, st>>>(ctx->partials, ctx->partials_used,
+                                                        max_norm, ctx->scalars);
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  ctx->norm_issued = true;
+  return SLIDEDP_OK;
+}
+
+// Copies the four scalars to the pinned mirror on `st` and waits (bounded) for them.
+static int fetch_scalars(slidedp_ctx* ctx, cudaStream_t st) {
+  CU(cudaMemcpyAsync(ctx->host_scalars, ctx->scalars, 4 * sizeof(double),
+                     cudaMemcpyDeviceToHost, st));
+  CU(cudaEventRecord(ctx->scalar_event, st));
+  return bounded_event_wait(ctx, ctx->scalar_event, kWaitSeconds);
+}
+
+
+}  // namespace host
+}  // namespace slidedp
+
+extern "C" {
+
+int slidedp_grad_norm(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                      double inv_R, int first_chunk, void* cuda_stream) {
+  if (!ctx || n < 0 || inv_R != inv_R) return SLIDEDP_ERR_INVALID_ARG;
+  GradPtrs gp;
+  int rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  return norm_chunk(ctx, gp, R, n, inv_R, first_chunk, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int slidedp_grad_norm_finish(slidedp_ctx* ctx, double max_norm, double* host_norm,
+                             double* host_coef, void* cuda_stream) {
+  if (!ctx || max_norm != max_norm) return SLIDEDP_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int rc = norm_finish(ctx, max_norm, st);
+  if (rc != SLIDEDP_OK) return rc;
+  if (host_norm || host_coef) {
+    rc = fetch_scalars(ctx, st);
+    if (rc != SLIDEDP_OK) return rc;
+    if (host_norm) *host_norm = ctx->host_scalars[1];
+    if (host_coef) *host_coef = ctx->host_scalars[2];
+  }
+  return SLIDEDP_OK;
+}
+
+int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                               float* master, float* m, float* v, void* param_bf16_out,
+                               const slidedp_hparams* hp, void* cuda_stream) {
+  if (!ctx || n < 0) return SLIDEDP_ERR_INVALID_ARG;
+  int rc = check_hparams(hp);
+  if (rc != SLIDEDP_OK) return rc;
+  GradPtrs gp;
+  rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  if (n > 0 && (!master || !m || !v || !param_bf16_out)) return SLIDEDP_ERR_INVALID_ARG;
+  if (!aligned16(master) || !aligned16(m) || !aligned16(v) || !aligned16(param_bf16_out))
+    return SLIDEDP_ERR_MISALIGNED;
+  const bool clip = hp->max_norm > 0.0;
+  if (clip && !ctx->norm_issued) return SLIDEDP_ERR_NO_NORM;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  return launch_update(ctx, gp, R, n, master, m, v, static_cast<uint16_t*>(param_bf16_out),
+                       make_consts(hp), clip ? ctx->scalars + 2 : nullptr,
+                       static_cast<cudaStream_t>(cuda_stream));
+}
+
+int slidedp_reduce_mean_bf16(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                             double inv_R, void* out_bf16, void* cuda_stream) {
+  if (!ctx || n < 0 || inv_R != inv_R) return SLIDEDP_ERR_INVALID_ARG;
+  GradPtrs gp;
+  int rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  if (n > 0 && !out_bf16) return SLIDEDP_ERR_INVALID_ARG;
+  if (!aligned16(out_bf16)) return SLIDEDP_ERR_MISALIGNED;
+  if (n == 0) return SLIDEDP_OK;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const unsigned blocks = (unsigned)((n + 8 * kReduceThreads - 1) / (8 * kReduceThreads));
+  uint16_t* out = static_cast<uint16_t*>(out_bf16);
+  const float inv = (float)inv_R;
+  switch (R) {
+#define SLIDEDP_CASE(r) \
+  case r: reduce_mean_bf16_kernel<r><<<blocks, kReduceThreads, 0, st>>>(gp, n, inv, out); break;
+    SLIDEDP_CASE(1) SLIDEDP_CASE(2) SLIDEDP_CASE(3) SLIDEDP_CASE(4) SLIDEDP_CASE(5) SLIDEDP_CASE(6)
+    SLIDEDP_CASE(7) SLIDEDP_CASE(8) SLIDEDP_CASE(9) SLIDEDP_CASE(10) SLIDEDP_CASE(11)
+    SLIDEDP_CASE(12) SLIDEDP_CASE(13) SLIDEDP_CASE(14) SLIDEDP_CASE(15) SLIDEDP_CASE(16)
+#undef SLIDEDP_CASE
+    default: return SLIDEDP_ERR_INVALID_ARG;
+  }
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  return SLIDEDP_OK;
+}
+
+// ---- norm without allocation ---------------------------------------------------------------
+//
+// Scratch for callers that cannot allocate: the per-tile sums live in an array that is part
+// of the library's device image. In HOST code the name `noalloc_tile_sums` is only a handle
+// for the symbol, not a device address; the address each device gave it is looked up once
+// per device with cudaGetSymbolAddress (with that device current) and cached here.
+constexpr int64_t kNoallocMaxTiles = SLIDEDP_NOALLOC_MAX_ELEMS / kNormTile;   // 65536
+static __device__ __align__(256) double noalloc_tile_sums[kNoallocMaxTiles];
+
+constexpr int kNoallocMaxDevices = 64;
+static double* noalloc_scratch_addr[kNoallocMaxDevices];   // zero-initialised: not looked up yet
+
+int slidedp_grad_norm_noalloc(const void* const* grads_bf16, int R, int64_t n, double inv_R,
+                              double max_norm, double* out4, void* cuda_stream) {
+  if (n < 0 || !out4 || inv_R != inv_R || max_norm != max_norm) return SLIDEDP_ERR_INVALID_ARG;
+  GradPtrs gp;
+  int rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  if (!aligned16(out4)) return SLIDEDP_ERR_MISALIGNED;
+  if (n > SLIDEDP_NOALLOC_MAX_ELEMS) return SLIDEDP_ERR_TOO_LARGE;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return SLIDEDP_ERR_CUDA; }
+  if (dev < 0 || dev >= kNoallocMaxDevices) return SLIDEDP_ERR_INVALID_ARG;
+  double* scratch = noalloc_scratch_addr[dev];
+  if (!scratch) {
+    // one-time set-up for this device (current right now): resolve the symbol's address
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, noalloc_tile_sums) != cudaSuccess || !p) {
+      (void)cudaGetLastError();
+      return SLIDEDP_ERR_CUDA;
+    }
+    scratch = static_cast<double*>(p);
+    noalloc_scratch_addr[dev] = scratch;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
+  if (ntiles > 0) {
+    const unsigned blocks = (unsigned)ntiles;
+    const float inv = (float)inv_R;
+    launch_sumsq(gp, R, n, inv, scratch, blocks, st);
+    if (cudaGetLastError() != cudaSuccess) return SLIDEDP_ERR_CUDA;
+  }
+  // reads tiles [0, ntiles) only: whatever an earlier call left beyond them is never seen
+  grad_norm_finish_kernel<<<1, kFinishThreads, 0, st>>>(scratch, ntiles, max_norm, out4);
+  if (cudaGetLastError() != cudaSuccess) return SLIDEDP_ERR_CUDA;
+  return SLIDEDP_OK;
+}
+
+}  // extern "C"

@@ -409,3 +409,21 @@ def test_rank_reduction_alone_returns_the_bf16_mean_bit_exact(ctx, sd, R):
         want = oracle.reduce_mean_bf16([parity.u16(x) for x in grads], 1.0 / R) if n else np.zeros(0, np.uint16)
         assert np.array_equal(parity.u16(out[:n]), want), (R, n)
         assert torch.all(out[n:] == 9.0)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_config2_shape_many_seeds_multi_step(ctx, sd, seed):
+    """The benchmark's hyper-parameters on a 3 M-parameter cut of the layer, eight seeds, three
+    consecutive clipped steps each, both sides restarted from the oracle's state every step so
+    that each step is a single-step comparison on realistic warm moments."""
+    import dataclasses
+    wl = dataclasses.replace(W.scaled(W.CONFIGS["qwen3_8b_layer"], 64), seed=100 + seed)
+    n, R = wl.numel, wl.R
+    w = parity.f32(W.master_weights(wl)).copy()
+    m, v = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    for t in range(1, 4):
+        grads = [W.rank_gradient(wl, r, step=t) for r in range(R)]
+        got, want = run_both(ctx, sd, grads, torch.from_numpy(w), torch.from_numpy(m),
+                             torch.from_numpy(v), dict(wl.hparams, step=t), 0.5)
+        assert_parity(f"seed {seed} step {t}", got, want, 0.5)
+        w, m, v = want[0], want[1], want[2]

@@ -29,6 +29,8 @@
  *    default stream). Device-resident calls only enqueue work on that stream and return.
  *  - master / m / v are updated in place; gradients are read-only; param_bf16_out must
  *    not overlap any other argument.
+ *  - A context is not thread-safe: use one per host thread, or serialise the calls on it. All
+ *    device pointers passed with a context must live on that context's device.
  */
 #ifndef SLIDEDP_H
 #define SLIDEDP_H

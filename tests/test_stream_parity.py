@@ -268,3 +268,32 @@ def test_zero_copy_update_on_pinned_host_state_matches_the_device_path(ctx, sd):
     for a, b in ((hw, w), (hm, m), (hv, v)):
         assert np.array_equal(a.numpy(), parity.f32(b))
     assert np.array_equal(parity.u16(zp), parity.u16(dp))
+
+
+@pytest.mark.parametrize("n", [1, 7, 8, 9, 1000, 4099])
+def test_tiny_and_ragged_host_resident_steps(ctx, sd, n):
+    """Host-resident steps far below one chunk, and with chunks of 8 and 16 elements: the slot
+    ring, the ragged tail and the norm all on the smallest sizes."""
+    R = 3
+    g = torch.Generator().manual_seed(70 + n)
+    grads = [(torch.randn(n, generator=g) * 1e-2).to(torch.bfloat16) for _ in range(R)]
+    w0 = (torch.randn(n, generator=g) * 0.02).numpy()
+    m0 = (torch.randn(n, generator=g) * 1e-3).numpy()
+    v0 = (torch.randn(n, generator=g).square() * 1e-6).numpy()
+    kw = dict(inv_R=1.0 / R, max_norm=0.01, step=6, lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8,
+              weight_decay=0.1)
+    ow, om, ov, op = w0.copy(), m0.copy(), v0.copy(), np.zeros(n, np.uint16)
+    norm_o, _ = oracle.step([parity.u16(x) for x in grads], ow, om, ov, op, oracle.HParams(**kw))
+    dg = [x.cuda() for x in grads]
+    for chunk, nbuf in ((8, 2), (16, 3), (1 << 20, 2)):
+        if n // chunk > 300:
+            continue
+        hw, hm, hv = pinned(w0), pinned(m0), pinned(v0)
+        dp = torch.zeros(max(n, 8), dtype=torch.bfloat16, device="cuda")
+        st = ctx.slidedp_stream_step(dg, n, hw, hm, hv, dp, chunk, nbuf, sd.HParams(**kw))
+        parity.assert_fp32_close(f"n={n}/master", hw.numpy(), ow)
+        parity.assert_fp32_close(f"n={n}/m", hm.numpy(), om)
+        parity.assert_fp32_close(f"n={n}/v", hv.numpy(), ov)
+        parity.assert_bf16_close(f"n={n}/param_bf16", parity.u16(dp[:n]), op)
+        parity.assert_norm_close(st["norm"], norm_o)
+        assert st["chunks"] == -(-n // chunk)

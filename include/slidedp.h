@@ -132,7 +132,10 @@ SLIDEDP_API int slidedp_grad_norm_finish(slidedp_ctx* ctx, double max_norm, doub
  *   w'   = w - lr * ( (m'/(1-beta1^t)) / (sqrt(v'/(1-beta2^t)) + eps) + weight_decay * w )
  *   master[i], m[i], v[i] = fl32(w'), fl32(m'), fl32(v')      (FP64 arithmetic, one rounding)
  *   param_bf16_out[i] = bf16_round_to_nearest_even(master[i])
- * grads_bf16: host array of R device pointers to n BF16 values each. master, m, v: device,
+ * grads_bf16: host array of R device pointers to n BF16 values each; a pointer may also address
+ * a peer GPU's buffer with peer access enabled (the kernel reads gradients with plain global
+ * loads in rank order, which is what fuses the cross-rank reduction into the update; no bulk or
+ * multicast copy is used). master, m, v: device,
  * n floats, in place. param_bf16_out: device, n BF16 values. When hp->max_norm > 0 a
  * slidedp_grad_norm_finish must have been enqueued earlier on the same stream
  * (SLIDEDP_ERR_NO_NORM if none was ever issued on this context).

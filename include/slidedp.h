@@ -121,6 +121,24 @@ SLIDEDP_API int slidedp_grad_norm(slidedp_ctx* ctx, const void* const* grads_bf1
 SLIDEDP_API int slidedp_grad_norm_finish(slidedp_ctx* ctx, double max_norm, double* host_norm /* nullable */,
                              double* host_coef /* nullable */, void* cuda_stream);
 
+/* The two halves of the norm with the tile sums in CALLER memory, for a step whose parameters are
+ * sharded over several GPUs (each GPU updates a contiguous shard and reads its slice of every
+ * rank's gradient, Sec. 3.2 "Parameter dispatch" / "Gradient return"): each GPU computes the tile
+ * sums of its shard with slidedp_grad_norm_tiles, the shards' sums are gathered in shard order
+ * into one array (an all-gather of 8 bytes per 16384 parameters), and every GPU folds that array
+ * with slidedp_grad_norm_finish_from. If the shard bounds are multiples of SLIDEDP_NORM_TILE
+ * elements the gathered array equals the tile sums of the unsharded step, so every GPU obtains
+ * bit for bit the coefficient of the single-GPU step.
+ * tile_sums_out: device, ceil(n / SLIDEDP_NORM_TILE) doubles. tile_sums: device, count doubles.
+ * slidedp_grad_norm_finish_from leaves norm and coefficient in the context exactly like
+ * slidedp_grad_norm_finish (same host_norm / host_coef behaviour). */
+#define SLIDEDP_NORM_TILE 16384
+SLIDEDP_API int slidedp_grad_norm_tiles(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                            double inv_R, double* tile_sums_out, void* cuda_stream);
+SLIDEDP_API int slidedp_grad_norm_finish_from(slidedp_ctx* ctx, const double* tile_sums, int64_t count,
+                                  double max_norm, double* host_norm /* nullable */,
+                                  double* host_coef /* nullable */, void* cuda_stream);
+
 /* ---- device-resident update: one fused kernel per chunk -------------------------------
  *
  * For i in [0, n):   (Sec. 3.2: one update of the authoritative FP32 state per iteration

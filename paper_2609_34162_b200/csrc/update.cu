@@ -142,6 +142,46 @@ int slidedp_grad_norm_finish(slidedp_ctx* ctx, double max_norm, double* host_nor
   return SLIDEDP_OK;
 }
 
+int slidedp_grad_norm_tiles(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                            double inv_R, double* tile_sums_out, void* cuda_stream) {
+  if (!ctx || n < 0 || inv_R != inv_R) return SLIDEDP_ERR_INVALID_ARG;
+  GradPtrs gp;
+  int rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  if (n == 0) return SLIDEDP_OK;
+  if (!tile_sums_out) return SLIDEDP_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(tile_sums_out) & 7u) != 0) return SLIDEDP_ERR_MISALIGNED;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
+  launch_sumsq(gp, R, n, (float)inv_R, tile_sums_out, (unsigned)ntiles,
+               static_cast<cudaStream_t>(cuda_stream));
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  return SLIDEDP_OK;
+}
+
+int slidedp_grad_norm_finish_from(slidedp_ctx* ctx, const double* tile_sums, int64_t count,
+                                  double max_norm, double* host_norm, double* host_coef,
+                                  void* cuda_stream) {
+  if (!ctx || count < 0 || max_norm != max_norm || (count > 0 && !tile_sums))
+    return SLIDEDP_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  grad_norm_finish_kernel<<<1, kFinishThreads, 0, st>>>(tile_sums, count, max_norm, ctx->scalars);
+  ctx->launches += 1;
+  CU(cudaGetLastError());
+  ctx->norm_issued = true;
+  if (host_norm || host_coef) {
+    int rc = fetch_scalars(ctx, st);
+    if (rc != SLIDEDP_OK) return rc;
+    if (host_norm) *host_norm = ctx->host_scalars[1];
+    if (host_coef) *host_coef = ctx->host_scalars[2];
+  }
+  return SLIDEDP_OK;
+}
+
 int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
                                float* master, float* m, float* v, void* param_bf16_out,
                                const slidedp_hparams* hp, void* cuda_stream) {

@@ -24,6 +24,7 @@ if not os.path.exists(LIB_PATH):
 _lib = ctypes.CDLL(LIB_PATH)
 
 MAX_RANKS = 16
+NORM_TILE = 16384
 OK, ERR_INVALID_ARG, ERR_MISALIGNED, ERR_BUDGET, ERR_NOT_PINNED, ERR_CUDA, ERR_TIMEOUT, ERR_NO_NORM = (
     0, -1, -2, -3, -4, -5, -6, -7)
 ERR_TOO_LARGE = -8
@@ -79,6 +80,12 @@ _lib.slidedp_grad_norm.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, ctype
 _lib.slidedp_grad_norm_finish.restype = ctypes.c_int
 _lib.slidedp_grad_norm_finish.argtypes = [_vp, ctypes.c_double, ctypes.POINTER(ctypes.c_double),
                                           ctypes.POINTER(ctypes.c_double), _vp]
+_lib.slidedp_grad_norm_tiles.restype = ctypes.c_int
+_lib.slidedp_grad_norm_tiles.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, ctypes.c_double, _vp, _vp]
+_lib.slidedp_grad_norm_finish_from.restype = ctypes.c_int
+_lib.slidedp_grad_norm_finish_from.argtypes = [_vp, _vp, ctypes.c_int64, ctypes.c_double,
+                                               ctypes.POINTER(ctypes.c_double),
+                                               ctypes.POINTER(ctypes.c_double), _vp]
 _lib.slidedp_reduce_adamw_chunk.restype = ctypes.c_int
 _lib.slidedp_reduce_adamw_chunk.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp,
                                             _vp, ctypes.POINTER(_HParams), _vp]
@@ -213,6 +220,22 @@ class Context:
         self._check(_lib.slidedp_grad_norm_finish(self._h, max_norm, None, None, _stream(stream)))
         return None
 
+    def slidedp_grad_norm_tiles(self, grads, n: int, inv_R: float, tile_sums_out, stream=None) -> None:
+        self._check(_lib.slidedp_grad_norm_tiles(self._h, _grad_array(grads), len(grads), n, inv_R,
+                                                 _ptr(tile_sums_out), _stream(stream)))
+
+    def slidedp_grad_norm_finish_from(self, tile_sums, count: int, max_norm: float,
+                                      fetch: bool = False, stream=None):
+        if fetch:
+            norm, coef = ctypes.c_double(), ctypes.c_double()
+            self._check(_lib.slidedp_grad_norm_finish_from(
+                self._h, _ptr(tile_sums), count, max_norm, ctypes.byref(norm), ctypes.byref(coef),
+                _stream(stream)))
+            return norm.value, coef.value
+        self._check(_lib.slidedp_grad_norm_finish_from(self._h, _ptr(tile_sums), count, max_norm,
+                                                       None, None, _stream(stream)))
+        return None
+
     def slidedp_reduce_adamw_chunk(self, grads, n: int, master, m, v, param_bf16_out,
                                    hp: HParams, stream=None) -> None:
         c = hp._c()
@@ -278,6 +301,19 @@ def slidedp_model_stream_step(n_total: int, R: int, chunk_elems: int, nbuf: int,
     if rc != OK:
         raise SlideDPError(rc)
     return lo.value, pred.value
+
+
+def shard_bounds(n: int, shards: int):
+    """Contiguous shard bounds [(lo, hi), ...] of a flat space of n parameters over `shards`
+    GPUs, every interior bound a multiple of NORM_TILE so that the shards' tile sums, gathered
+    in shard order, are the tile sums of the unsharded step (argument arithmetic only)."""
+    tiles = -(-n // NORM_TILE)
+    bounds, lo_tile = [], 0
+    for s in range(shards):
+        hi_tile = lo_tile + tiles // shards + (1 if s < tiles % shards else 0)
+        bounds.append((min(lo_tile * NORM_TILE, n), min(hi_tile * NORM_TILE, n)))
+        lo_tile = hi_tile
+    return bounds
 
 
 def slidedp_create(device: int = 0, gpu_budget_bytes: int = 0) -> Context:

@@ -115,3 +115,15 @@ def test_comparators():
     b = np.array([0x3F81, 0x8000, 0x0000, 0x7F7F], np.uint16)
     assert parity.bf16_mismatch(a, a) == (0, 0.0)
     assert parity.bf16_mismatch(a, b) == (1, 0.5)      # +0 and -0 coincide on the line
+
+
+def test_shard_bounds_are_tile_aligned_and_cover_the_space():
+    import paper_2609_34162_b200.slidedp as b
+    for n in (0, 1, 16383, 16384, 16385, 192_946_176, 2_642_493_440):
+        for shards in (1, 2, 3, 4, 8, 16):
+            bounds = b.shard_bounds(n, shards)
+            assert len(bounds) == shards and bounds[0][0] == 0 and bounds[-1][1] == n
+            assert all(x[1] == y[0] for x, y in zip(bounds, bounds[1:]))
+            assert all((lo % b.NORM_TILE == 0 or lo == n) and lo <= hi for lo, hi in bounds)
+            sizes = [hi - lo for lo, hi in bounds]
+            assert max(sizes) - min(sizes) <= 2 * b.NORM_TILE     # balanced to a tile

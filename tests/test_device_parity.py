@@ -427,3 +427,43 @@ def test_config2_shape_many_seeds_multi_step(ctx, sd, seed):
                              torch.from_numpy(v), dict(wl.hparams, step=t), 0.5)
         assert_parity(f"seed {seed} step {t}", got, want, 0.5)
         w, m, v = want[0], want[1], want[2]
+
+
+@pytest.mark.parametrize("shards", [2, 3, 4, 8])
+def test_sharded_step_emulated_on_one_gpu_is_bit_identical(ctx, sd, shards):
+    """The multi-GPU form of the step, emulated as one GPU doing every shard in turn: tile-aligned
+    shard bounds, per-shard tile sums written to one gathered array in shard order, the fold of
+    that array on "every GPU", and the fused update of each shard from all ranks' gradient slices.
+    Norm, coefficient, state and BF16 copy must equal the unsharded step bit for bit."""
+    n, R = 16384 * 19 + 777, 4
+    grads, w, m, v = random_case(n, R, seed=900 + shards, sigma=1e-2)
+    dg = [g.cuda() for g in grads]
+    hp = sd.HParams(inv_R=0.25, max_norm=0.5, step=3)
+    # unsharded reference
+    rw, rm, rv = w.cuda(), m.cuda(), v.cuda()
+    rp = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    ctx.slidedp_grad_norm(dg, n, 0.25, True)
+    ref = ctx.slidedp_grad_norm_finish(0.5, fetch=True)
+    ctx.slidedp_reduce_adamw_chunk(dg, n, rw, rm, rv, rp, hp)
+    # sharded
+    bounds = sd.shard_bounds(n, shards)
+    assert bounds[0][0] == 0 and bounds[-1][1] == n
+    assert all(a[1] == b[0] for a, b in zip(bounds, bounds[1:]))
+    assert all(lo % sd.NORM_TILE == 0 for lo, _ in bounds)
+    total_tiles = -(-n // sd.NORM_TILE)
+    gathered = torch.full((total_tiles,), float("nan"), dtype=torch.float64, device="cuda")
+    at = 0
+    for lo, hi in bounds:
+        ctx.slidedp_grad_norm_tiles([g[lo:] for g in dg], hi - lo, 0.25, gathered[at:])
+        at += -(-(hi - lo) // sd.NORM_TILE)
+    assert at == total_tiles
+    got = ctx.slidedp_grad_norm_finish_from(gathered, total_tiles, 0.5, fetch=True)
+    assert got == ref
+    sw, sm, sv = w.cuda(), m.cuda(), v.cuda()
+    sp = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    for lo, hi in reversed(bounds):                      # any order: shards are independent
+        ctx.slidedp_reduce_adamw_chunk([g[lo:] for g in dg], hi - lo, sw[lo:], sm[lo:], sv[lo:],
+                                       sp[lo:], hp)
+    torch.cuda.synchronize()
+    for a, b in ((sw, rw), (sm, rm), (sv, rv), (sp, rp)):
+        assert torch.equal(a, b)

@@ -274,7 +274,7 @@ def run_cuda(args):
                               "frac": 2 * R * n / (norm_ms * 1e-3) / 1e9 / peak}}
 
     # ---- e2e: the same step with the FP32 state in pinned host memory ------------------
-    ce = W.chunk_elems(64)
+    ce = W.chunk_elems(16)      # a 12-chunk layer at 64 MiB would spend 8 % draining the last chunk
     hw = torch.empty(n, pin_memory=True); hm = torch.empty(n, pin_memory=True)
     hv = torch.empty(n, pin_memory=True)
     hw.copy_(w); hm.copy_(m); hv.copy_(v)
@@ -295,7 +295,7 @@ def run_cuda(args):
     e2e = {"value": job_value(world, n, e2e_steps, e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": 12 * n, "d2h_bytes_per_step": 12 * n + 32,
            "ms_per_step": e2e_ms / e2e_steps, "wall_ms_per_step": wall / e2e_steps * 1e3,
-           "steps": e2e_steps, "chunk_mib": 64, "nbuf": 3,
+           "steps": e2e_steps, "chunk_mib": 16, "nbuf": 3,
            "note": "FP32 master/m/v in pinned host memory, copied H2D and back D2H every step; "
                    "gradients and the BF16 copy stay on the device where backward/forward use them",
            "link_gbs_h2d": last["gbs_h2d"], "link_gbs_d2h": last["gbs_d2h"]}

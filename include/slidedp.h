@@ -52,7 +52,8 @@ extern "C" {
 
 typedef enum {
   SLIDEDP_OK = 0,
-  SLIDEDP_ERR_INVALID_ARG = -1, /* null pointer, R outside 1..16, n < 0, step < 1, beta outside [0,1), ... */
+  SLIDEDP_ERR_INVALID_ARG = -1, /* null pointer, R outside 1..16, n < 0, step < 1, beta outside [0,1),
+                                   non-finite lr / eps / weight decay / 1/R, ...                        */
   SLIDEDP_ERR_MISALIGNED = -2,  /* a base pointer is not 16-byte aligned                               */
   SLIDEDP_ERR_BUDGET = -3,      /* the streaming slots would not fit the context's GPU memory budget   */
   SLIDEDP_ERR_NOT_PINNED = -4,  /* a host state pointer of slidedp_stream_step is not page-locked      */
@@ -79,7 +80,7 @@ typedef struct {
   double ms_total;        /* first enqueue to last D2H complete                                */
   double ms_norm;         /* the norm pass when it ran inside the call                         */
   double ms_h2d;          /* copy-in lane: start of its first copy to end of its last copy    */
-  double ms_kernel;       /* update kernels: the first chunk's kernel time scaled to n_total   */
+  double ms_kernel;       /* update kernels: the middle chunk's kernel time scaled to n_total  */
   double ms_d2h;          /* copy-out lane: start of its first copy to end of its last copy   */
   double gbs_h2d, gbs_d2h;/* bytes moved / that lane's span                                    */
   int64_t chunks;
@@ -94,6 +95,37 @@ typedef struct {
 SLIDEDP_API int slidedp_create(slidedp_ctx** out, int device, size_t gpu_budget_bytes);
 /* Waits (bounded) for the context's own streams, frees everything. NULL is a no-op. */
 SLIDEDP_API int slidedp_destroy(slidedp_ctx* ctx);
+
+/* ---- failure handling ------------------------------------------------------------------
+ *
+ * (Paper Sec. 3.3 "Completion and buffer reuse" is the only related passage: a buffer is reused
+ * only after the work that reads it completed, and a stalled consumer exerts backpressure. The
+ * library adds a bound on every host-side wait so that a stalled device never blocks a caller
+ * for ever.)
+ *
+ * Every host-side wait of the library is a poll with a deadline of `wait_seconds` (default 300;
+ * slidedp_set_wait_seconds changes it for this context, 0 < seconds <= 86400). When a wait runs
+ * out the entry point returns SLIDEDP_ERR_TIMEOUT. Nothing is cancelled: the queued copies and
+ * kernels keep running, the caller's buffers must stay valid, and a later slidedp_stream_wait
+ * (after raising the bound or simply later) returns SLIDEDP_OK once they are done, after which
+ * the context is as usable as before and the step's results are complete.
+ *
+ * SLIDEDP_ERR_CUDA from a streaming entry point (slidedp_stream_step, _async, slidedp_deliver_params,
+ * slidedp_link_probe) means a runtime call failed midway through enqueuing. Before returning, the
+ * entry point waits (bounded) for the part it had already queued, so no copy touches the
+ * caller's memory after the return, and restarts its slot ring; the context stays usable. The
+ * host state is then partly updated: chunks queued before the failure carry the new values, the
+ * others the old ones, so the caller must restore its own copy of the step's inputs before
+ * retrying. From a device-resident entry point SLIDEDP_ERR_CUDA from a failed launch means the
+ * kernel was not queued and the state is untouched.
+ *
+ * slidedp_test_fail_nth_call is a HOST-SIDE test hook (nothing on the GPU is made to fail): the
+ * nth guarded CUDA runtime call (or kernel launch) that the context issues from now on is not
+ * issued at all and is reported as failed with cudaErrorUnknown, so that every error path above
+ * can be exercised; nth <= 0 switches the hook off. The countdown stops at the failure.
+ */
+SLIDEDP_API int slidedp_set_wait_seconds(slidedp_ctx* ctx, double seconds);
+SLIDEDP_API int slidedp_test_fail_nth_call(slidedp_ctx* ctx, int64_t nth);
 SLIDEDP_API const char* slidedp_strerror(int status);
 SLIDEDP_API int slidedp_last_cuda_error(const slidedp_ctx* ctx);
 
@@ -152,8 +184,8 @@ SLIDEDP_API int slidedp_grad_norm_finish_from(slidedp_ctx* ctx, const double* ti
  *   param_bf16_out[i] = bf16_round_to_nearest_even(master[i])
  * grads_bf16: host array of R device pointers to n BF16 values each; a pointer may also address
  * a peer GPU's buffer with peer access enabled (the kernel reads gradients with plain global
- * loads in rank order, which is what fuses the cross-rank reduction into the update; no bulk or
- * multicast copy is used). master, m, v: device,
+ * loads in rank order, which is what fuses the cross-rank reduction into the update: plain
+ * global loads only). master, m, v: device,
  * n floats, in place. param_bf16_out: device, n BF16 values. When hp->max_norm > 0 a
  * slidedp_grad_norm_finish must have been enqueued earlier on the same stream
  * (SLIDEDP_ERR_NO_NORM if none was ever issued on this context).
@@ -291,13 +323,21 @@ SLIDEDP_API int slidedp_link_probe(slidedp_ctx* ctx, void* host_a, void* host_b,
  * finite (else 0.0). Asynchronous on cuda_stream.
  *
  * Limits and sharing: n <= SLIDEDP_NOALLOC_MAX_ELEMS (2^30); more gives
- * SLIDEDP_ERR_TOO_LARGE and nothing is launched. The array (512 KiB) is held by every GPU
- * that loads the library until the process exits. All calls on a device share it: two calls
- * whose kernels may overlap on the GPU (different streams without ordering) race on it; calls
- * ordered on one stream are safe. It keeps the previous call's tile sums, and nothing has to
- * start at zero: each call overwrites the tiles it then reads and reads no others.
- * The first call on each device looks up the array's device address (a one-time set-up with
- * that device current); make that first call before starting any stream capture.
+ * SLIDEDP_ERR_TOO_LARGE and nothing is launched. The array (512 KiB) is part of the library's
+ * device image: every GPU on which the library's device code gets loaded holds it until the
+ * process exits. All calls on a device share it: two calls whose kernels may overlap on the GPU
+ * (different streams without ordering) race on it; calls ordered on one stream are safe. It
+ * keeps the previous call's tile sums, and nothing has to start at zero: each call overwrites
+ * the tiles it then reads and reads no others.
+ *
+ * The FIRST call on each device is a set-up call: with that device current it looks up the
+ * array's device address. Under CUDA's default lazy module loading that look-up can be the
+ * moment the driver loads the library's device image (array included) onto the GPU, which
+ * takes device memory inside the driver. So make one call per device at start-up (n = 0 is
+ * enough), OUTSIDE any region in which allocation is forbidden and before any stream capture;
+ * every later call on that device allocates nothing (a GPU test checks that free device memory
+ * does not move across later calls). The look-up is cached per device in an atomic, so first
+ * calls from several host threads at once are safe.
  */
 #define SLIDEDP_NOALLOC_MAX_ELEMS ((int64_t)1 << 30)
 SLIDEDP_API int slidedp_grad_norm_noalloc(const void* const* grads_bf16, int R, int64_t n, double inv_R,

@@ -63,9 +63,13 @@ int check_hparams(const slidedp_hparams* hp) {
   if (hp->step < 1) return SLIDEDP_ERR_INVALID_ARG;
   if (!(hp->beta1 >= 0.0 && hp->beta1 < 1.0)) return SLIDEDP_ERR_INVALID_ARG;
   if (!(hp->beta2 >= 0.0 && hp->beta2 < 1.0)) return SLIDEDP_ERR_INVALID_ARG;
-  if (!(hp->eps >= 0.0) || hp->lr != hp->lr || hp->weight_decay != hp->weight_decay ||
-      hp->inv_R != hp->inv_R)
-    return SLIDEDP_ERR_INVALID_ARG;
+  // eps, lr, weight decay and 1/R must be finite numbers (NaN fails every comparison below)
+  const double big = 1.7976931348623157e308;
+  if (!(hp->eps >= 0.0 && hp->eps <= big)) return SLIDEDP_ERR_INVALID_ARG;
+  if (!(hp->lr >= -big && hp->lr <= big)) return SLIDEDP_ERR_INVALID_ARG;
+  if (!(hp->weight_decay >= -big && hp->weight_decay <= big)) return SLIDEDP_ERR_INVALID_ARG;
+  if (!(hp->inv_R >= -big && hp->inv_R <= big)) return SLIDEDP_ERR_INVALID_ARG;
+  if (hp->max_norm != hp->max_norm) return SLIDEDP_ERR_INVALID_ARG;
   return SLIDEDP_OK;
 }
 

@@ -32,6 +32,18 @@ size_t slidedp_state_bytes(int64_t n) {
 int slidedp_last_cuda_error(const slidedp_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
 int64_t slidedp_kernel_launches(const slidedp_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int slidedp_set_wait_seconds(slidedp_ctx* ctx, double seconds) {
+  if (!ctx || !(seconds > 0.0) || seconds > 86400.0) return SLIDEDP_ERR_INVALID_ARG;
+  ctx->wait_seconds = seconds;
+  return SLIDEDP_OK;
+}
+
+int slidedp_test_fail_nth_call(slidedp_ctx* ctx, int64_t nth) {
+  if (!ctx) return SLIDEDP_ERR_INVALID_ARG;
+  ctx->fail_countdown = nth > 0 ? nth : 0;
+  return SLIDEDP_OK;
+}
+
 int slidedp_create(slidedp_ctx** out, int device, size_t gpu_budget_bytes) {
   if (!out) return SLIDEDP_ERR_INVALID_ARG;
   *out = nullptr;
@@ -82,11 +94,12 @@ int slidedp_create(slidedp_ctx** out, int device, size_t gpu_budget_bytes) {
 int slidedp_destroy(slidedp_ctx* ctx) {
   if (!ctx) return SLIDEDP_OK;
   DeviceGuard guard(ctx->device);
+  ctx->fail_countdown = 0;
   int rc = SLIDEDP_OK;
   cudaStream_t own[3] = {ctx->s_in, ctx->s_compute, ctx->s_out};
   for (cudaStream_t s : own)
     if (s) {
-      int r = bounded_stream_wait(ctx, s, kWaitSeconds);
+      int r = bounded_stream_wait(ctx, s, ctx->wait_seconds);
       if (r != SLIDEDP_OK && rc == SLIDEDP_OK) rc = r;
     }
   for (cudaStream_t s : own) if (s) cudaStreamDestroy(s);

@@ -13,11 +13,11 @@
 namespace slidedp {
 namespace host {
 
-constexpr double kWaitSeconds = 300.0;         // bound on every host-side wait
+constexpr double kDefaultWaitSeconds = 300.0;  // default bound on every host-side wait
 constexpr int64_t kInitialPartials = 1 << 20;  // 8 MB: 2^20 tiles = 17 G parameters
 
 
-// Timing events of ONE kernel (the first chunk's). Per-chunk timing events, on the copy
+// Timing events of ONE kernel (the middle chunk's). Per-chunk timing events, on the copy
 // streams or the compute stream, sit on the chunk's H2D -> kernel -> D2H chain and cost
 // several percent of link bandwidth at 16 MiB chunks, so a step records a fixed handful.
 struct ChunkEvents {
@@ -32,6 +32,10 @@ struct slidedp_ctx {
   size_t budget = 0;
   int last_cuda = 0;
   int64_t launches = 0;
+  double wait_seconds = slidedp::host::kDefaultWaitSeconds;   // slidedp_set_wait_seconds
+  // host-side fault injection (slidedp_test_fail_nth_call): the countdown-th guarded runtime
+  // call from now is not issued and reports cudaErrorUnknown; <= 0: off
+  int64_t fail_countdown = 0;
   // norm workspace
   double* partials = nullptr;
   int64_t partials_cap = 0;
@@ -75,11 +79,26 @@ struct DeviceGuard {
 
 int cuda_fail(slidedp_ctx* ctx, cudaError_t e);
 
-// Returns SLIDEDP_ERR_CUDA (recording the error in ctx) when a runtime call fails.
-#define CU(call)                                            \
-  do {                                                      \
-    cudaError_t e_ = (call);                                \
-    if (e_ != cudaSuccess) return slidedp::host::cuda_fail(ctx, e_);       \
+// True when the host-side fault injection of `ctx` says that the next guarded call must fail.
+inline bool injected_failure(slidedp_ctx* ctx) {
+  return ctx && ctx->fail_countdown > 0 && --ctx->fail_countdown == 0;
+}
+
+// Returns SLIDEDP_ERR_CUDA (recording the error in ctx) when a runtime call fails. Under fault
+// injection the call is NOT issued and counts as failed with cudaErrorUnknown.
+#define CU(call)                                                                              \
+  do {                                                                                        \
+    cudaError_t e_ = slidedp::host::injected_failure(ctx) ? cudaErrorUnknown : (call);        \
+    if (e_ != cudaSuccess) return slidedp::host::cuda_fail(ctx, e_);                          \
+  } while (0)
+// A guarded point with no call of its own: placed before a kernel launch, so that an injected
+// failure stops the entry point before the kernel could change any state.
+#define FAULT_POINT() CU(cudaSuccess)
+// The check after a kernel launch: never injected (the kernel has been queued already).
+#define CU_AFTER_LAUNCH()                                                                     \
+  do {                                                                                        \
+    cudaError_t e_ = cudaGetLastError();                                                      \
+    if (e_ != cudaSuccess) return slidedp::host::cuda_fail(ctx, e_);                          \
   } while (0)
 
 // Bounded host-side waits: polls, never an unbounded block inside the driver.

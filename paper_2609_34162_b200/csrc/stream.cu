@@ -39,17 +39,40 @@ int is_pinned(slidedp_ctx* ctx, const void* p, bool* pinned) {
 // Waits (bounded) until nothing queued on the context's three streams is left running.
 int drain_streams(slidedp_ctx* ctx) {
   for (cudaStream_t st : {ctx->s_out, ctx->s_compute, ctx->s_in}) {
-    int rc = bounded_stream_wait(ctx, st, kWaitSeconds);
+    int rc = bounded_stream_wait(ctx, st, ctx->wait_seconds);
     if (rc != SLIDEDP_OK) return rc;
   }
   ctx->ring_busy = false;
   return SLIDEDP_OK;
 }
 
+// After an entry point failed midway through enqueuing: wait (bounded) for whatever it did queue,
+// so that no copy still touches the caller's memory once the error is returned, and restart the
+// slot ring from a clean state. The original status is what the caller gets; if even the drain
+// times out the ring stays marked busy and a later slidedp_stream_wait finishes the job.
+int abandon_queued(slidedp_ctx* ctx, int status) {
+  const int64_t keep = ctx->fail_countdown;
+  ctx->fail_countdown = 0;                 // the clean-up itself is never a fault point
+  const int last = ctx->last_cuda;
+  if (drain_streams(ctx) == SLIDEDP_OK) {
+    ctx->ring_next = 0;
+    ctx->ring_cap = 0;                     // forces a fresh layout (and event state) next time
+    ctx->ring_nbuf = 0;
+  }
+  ctx->last_cuda = last;
+  ctx->fail_countdown = keep;
+  return status;
+}
+
 // Validates and enqueues one host-resident step on the context's streams. The slot ring
 // carries over from call to call (slot index = running chunk count mod nbuf, every copy-in
 // waits for the slot's last copy-out), so consecutive calls overlap like the chunks of one
 // call; a call with another slot layout first drains what is queued.
+int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total, float* host_master,
+                   float* host_m, float* host_v, void* param_bf16_out, int64_t chunk_elems,
+                   int nbuf, int64_t cap, int norm_ready, const slidedp_hparams* hp,
+                   bool synchronous, bool timed, int64_t nchunks);
+
 int enqueue_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n_total,
                         float* host_master, float* host_m, float* host_v, void* param_bf16_out,
                         int64_t chunk_elems, int nbuf, int norm_ready, const slidedp_hparams* hp,
@@ -109,6 +132,20 @@ int enqueue_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
   }
 
   ctx->ring_busy = true;
+  rc = enqueue_chunks(ctx, gp, R, n_total, host_master, host_m, host_v, param_bf16_out,
+                      chunk_elems, nbuf, cap, norm_ready, hp, synchronous, timed, nchunks);
+  if (rc != SLIDEDP_OK) return abandon_queued(ctx, rc);
+  return SLIDEDP_OK;
+}
+
+// The enqueue proper (everything after the checks and the slot allocation). Any failure in
+// here leaves work queued; the caller cleans up with abandon_queued.
+int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total, float* host_master,
+                   float* host_m, float* host_v, void* param_bf16_out, int64_t chunk_elems,
+                   int nbuf, int64_t cap, int norm_ready, const slidedp_hparams* hp,
+                   bool synchronous, bool timed, int64_t nchunks) {
+  const bool clip = hp->max_norm > 0.0;
+  int rc = SLIDEDP_OK;
   if (synchronous) {
     CU(cudaEventRecord(ctx->ev_begin, ctx->s_compute));
     CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_begin, 0));
@@ -133,7 +170,7 @@ int enqueue_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
     float* sw = ctx->slots + (size_t)slot * 3 * cap;
     float* sm = sw + cap;
     float* sv = sm + cap;
-    ChunkEvents* te = (timed && c == 0) ? &ctx->timing[0] : nullptr;
+    ChunkEvents* te = (timed && c == nchunks / 2) ? &ctx->timing[0] : nullptr;
     // copy-in: the slot must have been drained by the copy-out that last used it (a no-op
     // for an event that was never recorded or has completed)
     CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_free[slot], 0));
@@ -192,7 +229,7 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
   if (rc != SLIDEDP_OK) return rc;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
-  rc = bounded_event_wait(ctx, ctx->ev_end, kWaitSeconds);
+  rc = bounded_event_wait(ctx, ctx->ev_end, ctx->wait_seconds);
   if (rc != SLIDEDP_OK) return rc;
   rc = drain_streams(ctx);
   if (rc != SLIDEDP_OK) return rc;
@@ -207,9 +244,11 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
     stats->chunks = nchunks;
     if (nchunks > 0) {
       const ChunkEvents& te = ctx->timing[0];
-      const int64_t first_len = n_total < chunk_elems ? n_total : chunk_elems;
+      // the timed kernel is the middle chunk's (warm, with copies running on both sides)
+      const int64_t mid_off = (nchunks / 2) * chunk_elems;
+      const int64_t mid_len = n_total - mid_off < chunk_elems ? n_total - mid_off : chunk_elems;
       CU(cudaEventElapsedTime(&ms, te.k_start, te.k_end));
-      stats->ms_kernel = (double)ms * ((double)n_total / (double)first_len);
+      stats->ms_kernel = (double)ms * ((double)n_total / (double)mid_len);
       CU(cudaEventElapsedTime(&ms, ctx->ev_in_first, ctx->ev_in_last));
       stats->ms_h2d = ms;
       CU(cudaEventElapsedTime(&ms, ctx->ev_out_first, ctx->ev_out_last));
@@ -278,6 +317,8 @@ int slidedp_deliver_params(slidedp_ctx* ctx, const float* host_master, int64_t n
   const int64_t nchunks = n_total == 0 ? 0 : (n_total + chunk_elems - 1) / chunk_elems;
   uint16_t* pout = static_cast<uint16_t*>(param_bf16_out);
 
+  ctx->ring_busy = true;
+  auto enqueue = [&]() -> int {
   CU(cudaEventRecord(ctx->ev_begin, ctx->s_compute));
   CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_begin, 0));
   for (int64_t c = 0; c < nchunks; ++c) {
@@ -295,16 +336,22 @@ int slidedp_deliver_params(slidedp_ctx* ctx, const float* host_master, int64_t n
     // cast
     CU(cudaStreamWaitEvent(ctx->s_compute, ctx->ev_loaded[slot], 0));
     const unsigned blocks = (unsigned)((len + 8 * kCastThreads - 1) / (8 * kCastThreads));
+    FAULT_POINT();
     cast_master_to_bf16_kernel<<<blocks, kCastThreads, 0, ctx->s_compute>>>(sw, len, pout + off);
     ctx->launches += 1;
-    CU(cudaGetLastError());
+    CU_AFTER_LAUNCH();
     CU(cudaEventRecord(ctx->ev_free[slot], ctx->s_compute));
   }
   CU(cudaEventRecord(ctx->ev_end, ctx->s_compute));
-  rc = bounded_event_wait(ctx, ctx->ev_end, kWaitSeconds);
+  return SLIDEDP_OK;
+  };
+  rc = enqueue();
+  if (rc != SLIDEDP_OK) return abandon_queued(ctx, rc);
+  rc = bounded_event_wait(ctx, ctx->ev_end, ctx->wait_seconds);
   if (rc != SLIDEDP_OK) return rc;
-  rc = bounded_stream_wait(ctx, ctx->s_in, kWaitSeconds);
+  rc = bounded_stream_wait(ctx, ctx->s_in, ctx->wait_seconds);
   if (rc != SLIDEDP_OK) return rc;
+  ctx->ring_busy = false;
   if (stats) {
     float ms = 0.f;
     CU(cudaEventElapsedTime(&ms, ctx->ev_begin, ctx->ev_end));
@@ -332,8 +379,14 @@ int slidedp_link_probe(slidedp_ctx* ctx, void* host_a, void* host_b, void* dev_a
     if (rc != SLIDEDP_OK) return rc;
     if (!pinned) return SLIDEDP_ERR_NOT_PINNED;
   }
-  cudaEvent_t a0, a1, b0, b1;
-  CU(cudaEventCreate(&a0)); CU(cudaEventCreate(&a1)); CU(cudaEventCreate(&b0)); CU(cudaEventCreate(&b1));
+  cudaEvent_t a0 = nullptr, a1 = nullptr, b0 = nullptr, b1 = nullptr;
+  auto destroy_events = [&]() {
+    for (cudaEvent_t ev : {a0, a1, b0, b1}) if (ev) cudaEventDestroy(ev);
+  };
+  for (cudaEvent_t* ev : {&a0, &a1, &b0, &b1}) {
+    const cudaError_t e = injected_failure(ctx) ? cudaErrorUnknown : cudaEventCreate(ev);
+    if (e != cudaSuccess) { destroy_events(); return cuda_fail(ctx, e); }
+  }
   int rc = SLIDEDP_OK;
   auto pieces = [&](bool h2d, cudaStream_t st) -> cudaError_t {
     for (size_t off = 0; off < bytes; off += copy_bytes) {
@@ -350,8 +403,8 @@ int slidedp_link_probe(slidedp_ctx* ctx, void* host_a, void* host_b, void* dev_a
   for (int mode = 0; mode < 3 && rc == SLIDEDP_OK; ++mode) {
     double best_in = 0.0, best_out = 0.0;
     for (int rep = 0; rep < reps + 1 && rc == SLIDEDP_OK; ++rep) {  // first pass warms up
-      cudaError_t e = cudaSuccess;
-      if (mode != 1) {
+      cudaError_t e = injected_failure(ctx) ? cudaErrorUnknown : cudaSuccess;
+      if (e == cudaSuccess && mode != 1) {
         e = cudaEventRecord(a0, ctx->s_in);
         if (e == cudaSuccess) e = pieces(true, ctx->s_in);
         if (e == cudaSuccess) e = cudaEventRecord(a1, ctx->s_in);
@@ -362,8 +415,8 @@ int slidedp_link_probe(slidedp_ctx* ctx, void* host_a, void* host_b, void* dev_a
         if (e == cudaSuccess) e = cudaEventRecord(b1, ctx->s_out);
       }
       if (e != cudaSuccess) { rc = cuda_fail(ctx, e); break; }
-      if (mode != 1) rc = bounded_event_wait(ctx, a1, kWaitSeconds);
-      if (rc == SLIDEDP_OK && mode != 0) rc = bounded_event_wait(ctx, b1, kWaitSeconds);
+      if (mode != 1) rc = bounded_event_wait(ctx, a1, ctx->wait_seconds);
+      if (rc == SLIDEDP_OK && mode != 0) rc = bounded_event_wait(ctx, b1, ctx->wait_seconds);
       if (rc != SLIDEDP_OK) break;
       float ms = 0.f;
       if (mode != 1 && cudaEventElapsedTime(&ms, a0, a1) == cudaSuccess && rep > 0 && ms > 0) {
@@ -379,14 +432,15 @@ int slidedp_link_probe(slidedp_ctx* ctx, void* host_a, void* host_b, void* dev_a
     if (mode == 1) out4[1] = best_out;
     if (mode == 2) { out4[2] = best_in; out4[3] = best_out; }
   }
-  cudaEventDestroy(a0); cudaEventDestroy(a1); cudaEventDestroy(b0); cudaEventDestroy(b1);
+  if (rc != SLIDEDP_OK) {
+    // leave nothing running on the caller's buffers (bounded; the status stays the first one)
+    const int last = ctx->last_cuda;
+    bounded_stream_wait(ctx, ctx->s_in, ctx->wait_seconds);
+    bounded_stream_wait(ctx, ctx->s_out, ctx->wait_seconds);
+    ctx->last_cuda = last;
+  }
+  destroy_events();
   return rc;
 }
-
-// ---- norm without allocation ---------------------------------------------------------------
-//
-// Scratch for callers that cannot allocate: the per-tile sums live in an array that is part
-// of the library's device image. In HOST code the name `noalloc_tile_sums` is only a handle
-// for the symbol, not a device address; the address each device gave it is looked up once
 
 }  // extern "C"

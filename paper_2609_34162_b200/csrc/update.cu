@@ -4,6 +4,8 @@
 #include "internal.h"
 #include "kernels.cuh"
 
+#include <atomic>
+
 using namespace slidedp;
 using namespace slidedp::host;
 
@@ -22,6 +24,7 @@ int launch_update(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, float*
                   float* v, uint16_t* p, const UpdateConsts& k, const double* coef,
                   cudaStream_t st) {
   if (n == 0) return SLIDEDP_OK;
+  FAULT_POINT();
   // one instantiation per rank count: the R loads are fully unrolled (a runtime-R loop over a
   // 16-entry register array ran at 4.0 TB/s for R = 3 against 6.4+ TB/s unrolled)
   switch (R) {
@@ -33,7 +36,7 @@ int launch_update(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, float*
     default: return SLIDEDP_ERR_INVALID_ARG;
   }
   ctx->launches += 1;
-  CU(cudaGetLastError());
+  CU_AFTER_LAUNCH();
   return SLIDEDP_OK;
 }
 
@@ -61,7 +64,7 @@ static int ensure_partials(slidedp_ctx* ctx, int64_t need, cudaStream_t st) {
   cudaError_t e = cudaMemcpyAsync(bigger, ctx->partials, (size_t)ctx->partials_used * sizeof(double),
                                   cudaMemcpyDeviceToDevice, st);
   if (e == cudaSuccess) {
-    int rc = bounded_stream_wait(ctx, st, kWaitSeconds);
+    int rc = bounded_stream_wait(ctx, st, ctx->wait_seconds);
     if (rc != SLIDEDP_OK) { cudaFree(bigger); return rc; }
   } else {
     cudaFree(bigger);
@@ -84,18 +87,20 @@ int norm_chunk(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, double in
   const unsigned blocks = (unsigned)ntiles;
   double* dst = ctx->partials + ctx->partials_used;
   const float inv = (float)inv_R;
+  FAULT_POINT();
   launch_sumsq(gp, R, n, inv, dst, blocks, st);
   ctx->launches += 1;
-  CU(cudaGetLastError());
+  CU_AFTER_LAUNCH();
   ctx->partials_used += ntiles;
   return SLIDEDP_OK;
 }
 
 int norm_finish(slidedp_ctx* ctx, double max_norm, cudaStream_t st) {
+  FAULT_POINT();
   grad_norm_finish_kernel<<<1, kFinishThreads, 0, st>>>(ctx->partials, ctx->partials_used,
                                                         max_norm, ctx->scalars);
   ctx->launches += 1;
-  CU(cudaGetLastError());
+  CU_AFTER_LAUNCH();
   ctx->norm_issued = true;
   return SLIDEDP_OK;
 }
@@ -105,7 +110,7 @@ static int fetch_scalars(slidedp_ctx* ctx, cudaStream_t st) {
   CU(cudaMemcpyAsync(ctx->host_scalars, ctx->scalars, 4 * sizeof(double),
                      cudaMemcpyDeviceToHost, st));
   CU(cudaEventRecord(ctx->scalar_event, st));
-  return bounded_event_wait(ctx, ctx->scalar_event, kWaitSeconds);
+  return bounded_event_wait(ctx, ctx->scalar_event, ctx->wait_seconds);
 }
 
 
@@ -154,10 +159,11 @@ int slidedp_grad_norm_tiles(slidedp_ctx* ctx, const void* const* grads_bf16, int
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
   const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
+  FAULT_POINT();
   launch_sumsq(gp, R, n, (float)inv_R, tile_sums_out, (unsigned)ntiles,
                static_cast<cudaStream_t>(cuda_stream));
   ctx->launches += 1;
-  CU(cudaGetLastError());
+  CU_AFTER_LAUNCH();
   return SLIDEDP_OK;
 }
 
@@ -169,9 +175,10 @@ int slidedp_grad_norm_finish_from(slidedp_ctx* ctx, const double* tile_sums, int
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  FAULT_POINT();
   grad_norm_finish_kernel<<<1, kFinishThreads, 0, st>>>(tile_sums, count, max_norm, ctx->scalars);
   ctx->launches += 1;
-  CU(cudaGetLastError());
+  CU_AFTER_LAUNCH();
   ctx->norm_issued = true;
   if (host_norm || host_coef) {
     int rc = fetch_scalars(ctx, st);
@@ -218,6 +225,7 @@ int slidedp_reduce_mean_bf16(slidedp_ctx* ctx, const void* const* grads_bf16, in
   const unsigned blocks = (unsigned)((n + 8 * kReduceThreads - 1) / (8 * kReduceThreads));
   uint16_t* out = static_cast<uint16_t*>(out_bf16);
   const float inv = (float)inv_R;
+  FAULT_POINT();
   switch (R) {
 #define SLIDEDP_CASE(r) \
   case r: reduce_mean_bf16_kernel<r><<<blocks, kReduceThreads, 0, st>>>(gp, n, inv, out); break;
@@ -228,7 +236,7 @@ int slidedp_reduce_mean_bf16(slidedp_ctx* ctx, const void* const* grads_bf16, in
     default: return SLIDEDP_ERR_INVALID_ARG;
   }
   ctx->launches += 1;
-  CU(cudaGetLastError());
+  CU_AFTER_LAUNCH();
   return SLIDEDP_OK;
 }
 
@@ -241,8 +249,10 @@ int slidedp_reduce_mean_bf16(slidedp_ctx* ctx, const void* const* grads_bf16, in
 constexpr int64_t kNoallocMaxTiles = SLIDEDP_NOALLOC_MAX_ELEMS / kNormTile;   // 65536
 static __device__ __align__(256) double noalloc_tile_sums[kNoallocMaxTiles];
 
+// One slot per device, written once. Atomic so that two host threads making their first call
+// at the same time both end up with the same (identical) address and no data race.
 constexpr int kNoallocMaxDevices = 64;
-static double* noalloc_scratch_addr[kNoallocMaxDevices];   // zero-initialised: not looked up yet
+static std::atomic<double*> noalloc_scratch_addr[kNoallocMaxDevices];   // zero-initialised
 
 int slidedp_grad_norm_noalloc(const void* const* grads_bf16, int R, int64_t n, double inv_R,
                               double max_norm, double* out4, void* cuda_stream) {
@@ -255,16 +265,18 @@ int slidedp_grad_norm_noalloc(const void* const* grads_bf16, int R, int64_t n, d
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return SLIDEDP_ERR_CUDA; }
   if (dev < 0 || dev >= kNoallocMaxDevices) return SLIDEDP_ERR_INVALID_ARG;
-  double* scratch = noalloc_scratch_addr[dev];
+  double* scratch = noalloc_scratch_addr[dev].load(std::memory_order_acquire);
   if (!scratch) {
-    // one-time set-up for this device (current right now): resolve the symbol's address
+    // one-time set-up for this device (current right now): resolve the symbol's address. With
+    // lazy module loading this is also where the driver loads the library's device image,
+    // array included, which is why the header asks for this call at start-up.
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, noalloc_tile_sums) != cudaSuccess || !p) {
       (void)cudaGetLastError();
       return SLIDEDP_ERR_CUDA;
     }
     scratch = static_cast<double*>(p);
-    noalloc_scratch_addr[dev] = scratch;
+    noalloc_scratch_addr[dev].store(scratch, std::memory_order_release);
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int64_t ntiles = (n + kNormTile - 1) / kNormTile;

@@ -112,6 +112,10 @@ _lib.slidedp_grad_norm_noalloc.argtypes = [_pp, ctypes.c_int, ctypes.c_int64, ct
                                            ctypes.c_double, _vp, _vp]
 _lib.slidedp_kernel_launches.restype = ctypes.c_int64
 _lib.slidedp_kernel_launches.argtypes = [_vp]
+_lib.slidedp_set_wait_seconds.restype = ctypes.c_int
+_lib.slidedp_set_wait_seconds.argtypes = [_vp, ctypes.c_double]
+_lib.slidedp_test_fail_nth_call.restype = ctypes.c_int
+_lib.slidedp_test_fail_nth_call.argtypes = [_vp, ctypes.c_int64]
 
 
 class _Rates(ctypes.Structure):
@@ -204,6 +208,15 @@ class Context:
 
     def slidedp_kernel_launches(self) -> int:
         return int(_lib.slidedp_kernel_launches(self._h))
+
+    def slidedp_set_wait_seconds(self, seconds: float) -> None:
+        self._check(_lib.slidedp_set_wait_seconds(self._h, seconds))
+
+    def slidedp_test_fail_nth_call(self, nth: int) -> None:
+        self._check(_lib.slidedp_test_fail_nth_call(self._h, nth))
+
+    def slidedp_last_cuda_error(self) -> int:
+        return int(_lib.slidedp_last_cuda_error(self._h))
 
     def slidedp_grad_norm(self, grads, n: int, inv_R: float, first_chunk: bool = True,
                           stream=None) -> None:

@@ -42,11 +42,28 @@ def test_state_bytes_is_16_per_parameter(lib):
     assert lib.slidedp_state_bytes(-5) == 0
 
 
+def declared_statuses():
+    """{name: value} of the slidedp_status enum, read from the header."""
+    text = open(os.path.join(ROOT, "include", "slidedp.h")).read()
+    body = re.search(r"typedef enum \{(.*?)\} slidedp_status;", text, re.S).group(1)
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    return {k: int(v) for k, v in re.findall(r"(SLIDEDP_\w+)\s*=\s*(-?\d+)", body)}
+
+
 def test_strerror_names_every_status(lib):
     lib.slidedp_strerror.restype = ctypes.c_char_p
-    seen = {lib.slidedp_strerror(s).decode() for s in range(0, -8, -1)}
-    assert len(seen) == 8 and "unknown status" not in seen
+    statuses = declared_statuses()
+    assert statuses["SLIDEDP_OK"] == 0 and len(statuses) >= 9
+    assert sorted(statuses.values()) == list(range(-(len(statuses) - 1), 1))     # dense, no gaps
+    seen = {lib.slidedp_strerror(v).decode() for v in statuses.values()}
+    assert len(seen) == len(statuses) and "unknown status" not in seen
+    assert lib.slidedp_strerror(min(statuses.values()) - 1).decode() == "unknown status"
     assert lib.slidedp_strerror(-99).decode() == "unknown status"
+    # the binding's constants are the header's
+    import paper_2609_34162_b200.slidedp as sd
+    for name, value in statuses.items():
+        short = name.replace("SLIDEDP_", "")
+        assert getattr(sd, short) == value, name
 
 
 def test_argument_errors_need_no_gpu(lib):

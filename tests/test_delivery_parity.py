@@ -36,6 +36,7 @@ def same_bf16(got: np.ndarray, want: np.ndarray) -> bool:
 def deliver(ctx, host, chunk, nbuf):
     n = host.numel()
     out = torch.full((max(n, 8),), 7.0, dtype=torch.bfloat16, device="cuda")
+    torch.cuda.synchronize()          # the fill ran on torch's stream, the library uses its own
     st = ctx.slidedp_deliver_params(host, n, out, chunk, nbuf)
     return parity.u16(out[:n]), st
 

@@ -341,6 +341,7 @@ def test_guard_bands_around_every_buffer_stay_intact(ctx, sd, n):
     # delivery cast into a banded output
     host = torch.empty(n, pin_memory=True); host.copy_(w)
     pfull.fill_(-7.0)
+    torch.cuda.synchronize()
     ctx.slidedp_deliver_params(host, n, p, 8, 2)
     assert torch.all(pfull[:pad] == -7.0) and torch.all(pfull[pad + n:] == -7.0)
     assert torch.equal(p, w.to(torch.bfloat16))

@@ -7,8 +7,12 @@ relative, is the bar; in practice the bits are equal).
 
 This file sorts last on purpose: a run that stops at the first failure has then already run
 every other test. It passes alone in a fresh process and after the other tests."""
+import numpy as np
 import pytest
 import torch
+
+import oracle
+import parity
 
 pytestmark = pytest.mark.gpu
 
@@ -44,6 +48,33 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point(sd):
         assert abs(coef - want_coef) <= 1e-6 * want_coef
         assert abs(sumsq - want_norm ** 2) <= 1e-6 * sumsq and nonfinite == 0.0
         assert (norm, coef) == (want_norm, want_coef)          # same tree, same bits
+        # and directly against the CPU oracle, at the tolerance of the other norm tests
+        S = oracle.grad_sumsq([parity.u16(x) for x in grads], 1.0 / R, 4)
+        coef_o, norm_o = oracle.clip_coef(S, max_norm)
+        parity.assert_norm_close(norm, norm_o)
+        assert abs(coef - coef_o) <= 1e-6 * coef_o and abs(sumsq - S) <= 2e-6 * S
+
+
+def test_calls_after_the_first_take_no_device_memory(sd):
+    """The point of the entry point: once the set-up call on this device has been made (it may
+    load the library's device image), further calls must not move the device's free memory.
+    Every buffer is created before the measurement, so torch's own allocator is quiet too."""
+    g = torch.Generator(device="cuda").manual_seed(7)
+    n, R = 16384 * 9 + 11, 3
+    grads = [(torch.randn(n, generator=g, device="cuda") * 1e-3).to(torch.bfloat16) for _ in range(R)]
+    out = torch.zeros(4, dtype=torch.float64, device="cuda")
+    sd.slidedp_grad_norm_noalloc(grads, 0, 1.0 / R, 1.0, out)       # set-up call, n = 0
+    torch.cuda.synchronize()
+    assert out.tolist() == [0.0, 0.0, 1.0, 0.0]
+    torch.cuda.mem_get_info()
+    free_before, _ = torch.cuda.mem_get_info()
+    seen = set()
+    for _ in range(5):
+        sd.slidedp_grad_norm_noalloc(grads, n, 1.0 / R, 1.0, out)
+        torch.cuda.synchronize()
+        seen.add(tuple(out.tolist()))
+        assert torch.cuda.mem_get_info()[0] == free_before
+    assert len(seen) == 1 and next(iter(seen))[1] > 0.0              # and the same bits every time
 
 
 def test_limits_and_argument_errors(sd):

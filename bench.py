@@ -10,7 +10,12 @@ pass over all gradients, then the fused rank-reduce + AdamW + BF16-emit kernel.
 `value` is whole-job G-params/s with everything resident in HBM; `e2e` is the same step
 through slidedp_stream_step with the FP32 state in pinned HOST memory, host<->device copies
 inside the timed region. With --gpus N every rank updates its own layer (independent
-partitions, no data-path collective): weak scaling. Prints ONE JSON line on rank 0.
+partitions, no data-path collective): weak scaling. Under a launcher (torchrun) the ranks are the
+launcher's; without one, --gpus N > 1 starts the N ranks itself. Prints ONE JSON line on rank 0.
+
+  python bench.py --sharded --gpus N          # one layer sharded over N ranks (peer-mapped buffers)
+  python bench.py --report sweep              # the other configurations and the by-R table
+  python bench.py --report kernel --kernel update --params 50331648 --R 4   # one small case for ncu
 """
 from __future__ import annotations
 
@@ -178,8 +183,8 @@ def run_cuda(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: libslidedp has no CPU path "
+    if not torch.cuda.is_available() or local >= torch.cuda.device_count():
+        raise SystemExit("bench.py needs a CUDA device per rank: libslidedp has no CPU path "
                          "(use --impl reference for the CPU oracle)")
     torch.cuda.set_device(local)
     # under a launcher (torchrun sets RANK and MASTER_ADDR) the process group is used even for
@@ -332,6 +337,84 @@ def run_cuda(args):
     return 0
 
 
+def run_sharded(args):
+    """`--sharded`: ONE Qwen3-8B-shaped layer updated by all ranks together. Every rank holds its
+    own rank-local BF16 gradient of the whole layer (R = number of ranks), owns 1/N of the FP32
+    state, reads its slice of every peer's gradient through mapped pointers inside the norm and
+    update kernels, and stores its shard of the BF16 copy into every rank's parameter buffer
+    (paper_2609_34162_b200/sharded.py). Strong scaling: the layer is fixed, the ranks split it.
+    The timed region includes the three host-side barriers of each step."""
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_34162_b200.slidedp as sd
+    from paper_2609_34162_b200 import workloads as W
+    from paper_2609_34162_b200.sharded import ShardedStep
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available() or local >= torch.cuda.device_count():
+        raise SystemExit("bench.py --sharded needs one CUDA device per rank: libslidedp has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if "MASTER_ADDR" not in os.environ:
+        os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(_free_port()))
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    wl = W.CONFIGS[WORKLOAD]
+    n, R = wl.numel, world
+    ctx = sd.slidedp_create(local, 0)
+    grad = W.rank_gradient(wl, rank, step=wl.first_step, device=dev)
+    param = torch.zeros(n, dtype=torch.bfloat16, device=dev)
+    sh = ShardedStep(ctx, [grad], n, param)
+    lo, hi = sh.bounds[rank]
+    w = W.master_weights(wl, device=dev)[lo:hi].clone()
+    m, v = torch.zeros(hi - lo, device=dev), torch.zeros(hi - lo, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def hp(t):
+        return sd.HParams(inv_R=1.0 / R, max_norm=wl.max_norm, step=t, **wl.hparams)
+
+    t = 1
+    for _ in range(max(args.warmup, 3)):
+        sh.step(w, m, v, hp(t), stream)
+        t += 1
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = ctx.slidedp_kernel_launches()
+    dist.barrier(); torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record(stream)
+    for _ in range(args.steps):
+        sh.step(w, m, v, hp(t), stream)
+        t += 1
+    stop.record(stream)
+    dist.barrier(); torch.cuda.synchronize()
+    launches = ctx.slidedp_kernel_launches() - launches0
+    total_ms = max_over_ranks(start.elapsed_time(stop), world)
+    clocks = sampler.stop() if rank == 0 else None
+    sh.close()
+    ctx.slidedp_destroy()
+    if rank == 0:
+        # per parameter and rank: (12 + 14)/N state bytes locally, 2 (R - 1)/N gradient bytes
+        # and 2 (N - 1)/N parameter bytes over the GPU interconnect, plus the norm's re-read
+        print(json.dumps({
+            "metric": METRIC, "value": n * args.steps / (total_ms * 1e-3) / 1e9, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "mode": "sharded",
+            "config": {"workload": WORKLOAD, "params": n, "R": R, "clip_max_norm": wl.max_norm,
+                       "parallelism": f"one layer sharded over {world} rank(s): peer-mapped gradient "
+                                      "reads, BF16 copy stored to every rank, host barriers"},
+            "gpu_launches": launches, "clocks": clocks,
+            "interconnect_bytes_per_rank_per_step": (4 * (R - 1) + 2 * (world - 1)) * (hi - lo)}))
+    dist.barrier()
+    dist.destroy_process_group()
+    return 0
+
+
 def run_sweep(args):
     """`--report sweep`: one JSON line with the other benchmark configurations on one GPU:
     the tiny chunk (L2-resident and rotating over buffer sets larger than L2), the chunk-size
@@ -387,6 +470,51 @@ def run_sweep(args):
                    "(4 x L2) between reuses, the resident case is a cache number, not HBM")
     out["tiny"] = res
     del bufs
+
+    # ---- by rank count: update kernel, norm pass, rank reduction alone (100 M parameters)
+    n = 100_000_000
+    gen = torch.Generator(device=dev).manual_seed(11)
+    pool = [(torch.randn(n, generator=gen, device=dev) * 1e-3).to(torch.bfloat16) for _ in range(16)]
+    w = torch.randn(n, generator=gen, device=dev) * 0.02
+    m = torch.randn(n, generator=gen, device=dev) * 3e-4
+    v = torch.randn(n, generator=gen, device=dev).square() * 1e-7
+    p = torch.zeros(n, dtype=torch.bfloat16, device=dev)
+    by_R = []
+    reps = 12
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        for i in range(reps):
+            evs[i].record(st)
+            fn()
+        evs[reps].record(st)
+        torch.cuda.synchronize()
+        ms = sorted(evs[i].elapsed_time(evs[i + 1]) for i in range(reps))
+        return statistics.median(ms), ms[0]
+
+    for R in (1, 2, 3, 4, 8, 16):
+        g = pool[:R]
+        h = sd.HParams(inv_R=1.0 / R, max_norm=1.0, step=11)
+        ctx.slidedp_grad_norm(g, n, 1.0 / R, True)
+        ctx.slidedp_grad_norm_finish(1.0)
+
+        def norm_pass():
+            ctx.slidedp_grad_norm(g, n, 1.0 / R, True)
+            ctx.slidedp_grad_norm_finish(1.0)
+        row = {"R": R}
+        for name, fn, per in (("update", lambda: ctx.slidedp_reduce_adamw_chunk(g, n, w, m, v, p, h), 26 + 2 * R),
+                              ("norm", norm_pass, 2 * R),
+                              ("reduce_mean_bf16", lambda: ctx.slidedp_reduce_mean_bf16(g, n, 1.0 / R, p), 2 * R + 2)):
+            med, best = timed(fn)
+            row[name] = {"ms": med, "ms_best": best, "bytes_per_param": per,
+                         "gbs": per * n / (med * 1e6), "frac_of_measured_peak": per * n / (med * 1e6) / peak}
+        by_R.append(row)
+    out["by_rank_count"] = {"params": n, "timing": f"median of {reps} launches, CUDA events, inputs >> L2",
+                            "rows": by_R}
+    del pool, w, m, v, p
+    torch.cuda.empty_cache()
 
     def pinned_state(n):
         return [torch.empty(n, pin_memory=True) for _ in range(3)]
@@ -596,19 +724,123 @@ def cpu_baseline(W, torch, np, wl, grads, layer):
             "single_thread_sample": f"one whole step over the first {k} parameters"}
 
 
-def main():
+def run_kernel_case(args):
+    """`--report kernel`: a small, self-ending run of ONE kernel, for profiling under ncu
+    (inputs larger than the 126 MB L2 so DRAM counters mean something, but about a GB):
+
+      python bench.py --report kernel --kernel update --params 50331648 --R 4 --launches 4
+
+    Kernels: update (fused reduce + AdamW + BF16 emit), norm (tile sums + finish), reduce (rank
+    reduction alone), stream (host-resident step through pinned memory)."""
+    import torch
+
+    import paper_2609_34162_b200.slidedp as sd
+    n, R = args.params, args.R
+    dev = torch.device("cuda", 0)
+    g = torch.Generator(device=dev).manual_seed(0)
+    grads = [(torch.randn(n, generator=g, device=dev) * 1e-3).to(torch.bfloat16) for _ in range(R)]
+    w = torch.randn(n, generator=g, device=dev) * 0.02
+    m = torch.randn(n, generator=g, device=dev) * 3e-4
+    v = torch.randn(n, generator=g, device=dev).square() * 1e-7
+    p = torch.zeros(n, dtype=torch.bfloat16, device=dev)
+    ctx = sd.slidedp_create(0, 0)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.launches + 1)]
+    st = torch.cuda.current_stream()
+    if args.kernel == "stream":
+        hw, hm, hv = (torch.empty(n, pin_memory=True) for _ in range(3))
+        hw.copy_(w); hm.copy_(m); hv.copy_(v)
+    ctx.slidedp_grad_norm(grads, n, 1.0 / R, True)
+    ctx.slidedp_grad_norm_finish(args.clip)
+    torch.cuda.synchronize()
+    for i in range(args.launches):
+        ev[i].record(st)
+        hp = sd.HParams(inv_R=1.0 / R, max_norm=args.clip, step=11 + i)
+        if args.kernel == "update":
+            ctx.slidedp_reduce_adamw_chunk(grads, n, w, m, v, p, hp)
+        elif args.kernel == "norm":
+            ctx.slidedp_grad_norm(grads, n, 1.0 / R, True)
+            ctx.slidedp_grad_norm_finish(args.clip)
+        elif args.kernel == "reduce":
+            ctx.slidedp_reduce_mean_bf16(grads, n, 1.0 / R, p)
+        else:
+            ctx.slidedp_stream_step(grads, n, hw, hm, hv, p, 16 << 20, 3, hp, want_stats=False)
+    ev[args.launches].record(st)
+    torch.cuda.synchronize()
+    ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.launches)]
+    per = {"update": 26 + 2 * R, "norm": 2 * R, "reduce": 2 * R + 2, "stream": 24}[args.kernel]
+    print(json.dumps({"report": "kernel", "kernel": args.kernel, "params": n, "R": R,
+                      "ms_per_launch": ms, "bytes_per_param": per,
+                      "best_gbs": per * n / (min(ms) * 1e6)}))
+    ctx.slidedp_destroy()
+    return 0
+
+
+# ------------------------------------------------------------------- launching the ranks
+def _free_port() -> int:
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _rank_entry(rank, world, port, worker, args):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    sys.exit(worker(args))
+
+
+def launch_ranks(world: int, worker, args) -> int:
+    """Runs `worker(args)` as `world` processes of this node, one per GPU, with the launcher
+    environment (RANK, LOCAL_RANK, WORLD_SIZE, MASTER_ADDR = 127.0.0.1, MASTER_PORT) set as an
+    outer launcher would set it. Returns the first non-zero exit code, else 0."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    port = _free_port()
+    procs = [ctx.Process(target=_rank_entry, args=(r, world, port, worker, args))
+             for r in range(world)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join()
+    for p in procs:
+        if p.exitcode != 0:
+            return p.exitcode if p.exitcode and p.exitcode > 0 else 1
+    return 0
+
+
+def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
-    ap.add_argument("--report", choices=["contract", "sweep"], default="contract")
-    args = ap.parse_args()
+    ap.add_argument("--report", choices=["contract", "sweep", "kernel"], default="contract")
+    ap.add_argument("--sharded", action="store_true",
+                    help="one layer sharded over the ranks (peer-mapped gradients, BF16 copy stored "
+                         "to every rank) instead of one independent layer per rank")
+    ap.add_argument("--kernel", choices=["update", "norm", "reduce", "stream"], default="update")
+    ap.add_argument("--params", type=int, default=48 << 20)
+    ap.add_argument("--R", type=int, default=4)
+    ap.add_argument("--launches", type=int, default=4)
+    ap.add_argument("--clip", type=float, default=1.0)
+    args = ap.parse_args(argv)
+    if args.gpus < 1:
+        ap.error("--gpus must be at least 1")
+    launched = "RANK" in os.environ and "WORLD_SIZE" in os.environ
+    if launched and int(os.environ["WORLD_SIZE"]) != args.gpus:
+        print(f"bench.py: --gpus {args.gpus} disagrees with WORLD_SIZE={os.environ['WORLD_SIZE']} "
+              "set by the launcher", file=sys.stderr)
+        return 2
     if args.impl == "reference":
         return run_reference(args)
     if args.report == "sweep":
         return run_sweep(args)
-    return run_cuda(args)
+    if args.report == "kernel":
+        return run_kernel_case(args)
+    worker = run_sharded if args.sharded else run_cuda
+    if not launched and args.gpus > 1:
+        return launch_ranks(args.gpus, worker, args)      # no outer launcher: start the ranks here
+    return worker(args)
 
 
 if __name__ == "__main__":

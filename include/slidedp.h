@@ -198,6 +198,63 @@ SLIDEDP_API int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* 
                                float* master, float* m, float* v, void* param_bf16_out,
                                const slidedp_hparams* hp, void* cuda_stream);
 
+/* ---- the sharded multi-GPU step: buffers shared between processes, BF16 copy to every GPU ----
+ *
+ * With real ranks (one process per GPU, each holding its rank-local BF16 gradient of the whole
+ * layer) the step shards over the flat parameter space (paper Sec. 3.2: "Gradient return" sums
+ * the rank-local gradients and returns one result; "Parameter dispatch", sharded delivery, has
+ * every rank hold P_l/R of the layer and reconstructs it with an all-gather). GPU s owns the
+ * contiguous shard [lo_s, hi_s) of master / m / v and
+ *   1. reads slice [lo_s, hi_s) of EVERY rank's gradient through pointers mapped from the peers
+ *      (the kernels above read gradients with plain global loads in rank order, so the
+ *      cross-rank reduction is fused into the norm and update kernels and crosses the GPU
+ *      interconnect exactly once);
+ *   2. computes the tile sums of its shard (slidedp_grad_norm_tiles); the shards' sums are
+ *      gathered in shard order (8 bytes per 16384 parameters; slidedp_scatter_tile_sums stores
+ *      them straight into every GPU's gathered array) and folded by every GPU with
+ *      slidedp_grad_norm_finish_from, giving the coefficient of the unsharded step bit for bit
+ *      when the shard bounds are multiples of SLIDEDP_NORM_TILE;
+ *   3. updates its shard with slidedp_reduce_adamw_chunk_bcast, which is
+ *      slidedp_reduce_adamw_chunk with the BF16 copy stored into n_outs buffers instead of one:
+ *      the position of the shard in this GPU's BF16 parameter buffer and in every peer's
+ *      (mapped). The all-gather of the BF16 parameters is thus done by the update kernel's own
+ *      stores. param_bf16_outs: host array of n_outs (1..16) device pointers, each to n BF16
+ *      values, 16-byte aligned, none overlapping any other argument. Every other argument,
+ *      check, status and the arithmetic are those of slidedp_reduce_adamw_chunk (same bits).
+ * Ordering between GPUs is the caller's: a peer's buffer may be read (gradients) only after
+ * that peer has produced it, and written (BF16 copy) only when that peer no longer reads the
+ * previous copy; a peer sees the new copy after this GPU's stream has completed (a host-side
+ * barrier around the step does all three). paper_2609_34162_b200/sharded.py is the reference
+ * orchestration over torch.distributed.
+ *
+ * slidedp_ipc_export fills `out` for a caller-owned device buffer (any address inside a
+ * cudaMalloc'd allocation, e.g. a torch tensor of the default allocator; memory from
+ * virtual-memory-management allocators cannot be exported); the 80 bytes are plain data to send
+ * to the peer process by any means. slidedp_ipc_open maps a peer's handle into this process and
+ * returns the device address that corresponds to the exported one (valid on this context's
+ * device, peer access enabled on demand; a handle cannot be opened by the process that
+ * exported it). slidedp_ipc_close unmaps it (the context also unmaps what is left at destroy).
+ * The exporting process must keep the buffer allocated while a peer has it mapped.
+ */
+typedef struct {
+  unsigned char opaque[64]; /* the CUDA inter-process handle of the containing allocation */
+  uint64_t offset;          /* of the exported address inside that allocation             */
+  uint64_t bytes;           /* from the exported address to the end of the allocation     */
+} slidedp_ipc_handle;
+SLIDEDP_API int slidedp_ipc_export(slidedp_ctx* ctx, const void* dev_ptr, slidedp_ipc_handle* out);
+SLIDEDP_API int slidedp_ipc_open(slidedp_ctx* ctx, const slidedp_ipc_handle* handle, void** dev_ptr_out);
+SLIDEDP_API int slidedp_ipc_close(slidedp_ctx* ctx, void* dev_ptr);
+/* Step 2's gather without a collective library: stores this GPU's `count` tile sums
+ * (device, as written by slidedp_grad_norm_tiles) at dsts[0..n_dsts), each a device pointer to the
+ * position of this shard inside a GPU's gathered array (this GPU's own and the peers', mapped).
+ * Plain stores from one small kernel; asynchronous on cuda_stream. */
+SLIDEDP_API int slidedp_scatter_tile_sums(slidedp_ctx* ctx, const double* tile_sums, int64_t count,
+                              double* const* dsts, int n_dsts, void* cuda_stream);
+SLIDEDP_API int slidedp_reduce_adamw_chunk_bcast(slidedp_ctx* ctx, const void* const* grads_bf16, int R,
+                                     int64_t n, float* master, float* m, float* v,
+                                     void* const* param_bf16_outs, int n_outs,
+                                     const slidedp_hparams* hp, void* cuda_stream);
+
 /* ---- rank reduction alone ---------------------------------------------------------------------
  *
  * The paper's GPU-reduction route (Sec. 3.2 "Gradient return"): the rank-local gradients are summed,

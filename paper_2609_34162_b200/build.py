@@ -13,7 +13,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libslidedp.so")
 SOURCES = [os.path.join(CSRC, f) for f in ("common.cu", "context.cu", "update.cu", "stream.cu",
-                                           "model.cu")]
+                                           "model.cu", "ipc.cu")]
 DEPENDS = SOURCES + [os.path.join(CSRC, f) for f in ("kernels.cuh", "cast_kernel.cuh",
                                                      "device_utils.cuh", "types.h", "internal.h")]
 DEPENDS.append(os.path.join(ROOT, "include", "slidedp.h"))

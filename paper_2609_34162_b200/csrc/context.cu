@@ -108,6 +108,8 @@ int slidedp_destroy(slidedp_ctx* ctx) {
   kill(ctx->ev_in_first); kill(ctx->ev_in_last); kill(ctx->ev_out_first); kill(ctx->ev_out_last);
   for (int i = 0; i < 3; ++i) { kill(ctx->ev_loaded[i]); kill(ctx->ev_updated[i]); kill(ctx->ev_free[i]); }
   for (ChunkEvents& c : ctx->timing) { kill(c.k_start); kill(c.k_end); }
+  for (slidedp::host::IpcMapping& m : ctx->ipc) cudaIpcCloseMemHandle(m.base);
+  ctx->ipc.clear();
   if (ctx->slots) cudaFree(ctx->slots);
   if (ctx->partials) cudaFree(ctx->partials);
   if (ctx->scalars) cudaFree(ctx->scalars);

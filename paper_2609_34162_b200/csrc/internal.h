@@ -24,6 +24,14 @@ struct ChunkEvents {
   cudaEvent_t k_start, k_end;
 };
 
+// A peer process's allocation mapped into this process (slidedp_ipc_open).
+struct IpcMapping {
+  unsigned char opaque[64];
+  char* base;
+  size_t bytes;
+  int refs;
+};
+
 }  // namespace host
 }  // namespace slidedp
 
@@ -58,6 +66,7 @@ struct slidedp_ctx {
   cudaEvent_t ev_begin = nullptr, ev_norm_done = nullptr, ev_end = nullptr;
   cudaEvent_t ev_in_first = nullptr, ev_in_last = nullptr, ev_out_first = nullptr, ev_out_last = nullptr;
   std::vector<slidedp::host::ChunkEvents> timing;  // grown on demand, reused
+  std::vector<slidedp::host::IpcMapping> ipc;      // peer allocations mapped by slidedp_ipc_open
 };
 
 namespace slidedp {

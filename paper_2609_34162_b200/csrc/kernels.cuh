@@ -78,12 +78,36 @@ __device__ __forceinline__ void adamw_element(float gbar, float& w, float& m, fl
 // for a bulk-copy (TMA) shared-memory ring.
 // R is a template parameter (one instantiation per rank count 1..16): the R loads and the
 // left-to-right FP32 adds are fully unrolled.
-template <int R>
-__global__ void __launch_bounds__(kUpdateThreads, 8)
-reduce_adamw_kernel(GradPtrs gp, int64_t n, float* __restrict__ master,
-                    float* __restrict__ mom1, float* __restrict__ mom2,
-                    uint16_t* __restrict__ param_out, UpdateConsts k,
-                    const double* __restrict__ clip_coef) {
+//
+// Where the BF16 copy goes is a policy: OneOut stores it once (the single-GPU step); ManyOuts
+// stores the same values into several buffers, which in a sharded multi-GPU step are this
+// GPU's parameter buffer and every peer's, mapped into this process: the all-gather of the
+// BF16 parameters then happens inside the update kernel as plain peer stores, tile by tile.
+struct OneOut {
+  uint16_t* p;
+  __device__ __forceinline__ void vec(int64_t base, uint2 packed) const {
+    __stcs(reinterpret_cast<uint2*>(p + base), packed);
+  }
+  __device__ __forceinline__ void one(int64_t i, uint16_t bits) const { p[i] = bits; }
+};
+struct ManyOuts {
+  uint16_t* p[kMaxRanks];
+  int count;
+  __device__ __forceinline__ void vec(int64_t base, uint2 packed) const {
+    for (int o = 0; o < count; ++o) __stcs(reinterpret_cast<uint2*>(p[o] + base), packed);
+  }
+  __device__ __forceinline__ void one(int64_t i, uint16_t bits) const {
+    for (int o = 0; o < count; ++o) p[o][i] = bits;
+  }
+};
+
+template <int R, class Out>
+__device__ __forceinline__ void reduce_adamw_body(const GradPtrs& gp, int64_t n,
+                                                  float* __restrict__ master,
+                                                  float* __restrict__ mom1,
+                                                  float* __restrict__ mom2, const Out& out,
+                                                  const UpdateConsts& k,
+                                                  const double* __restrict__ clip_coef) {
   const int64_t base = ((int64_t)blockIdx.x * kUpdateThreads + threadIdx.x) * kVec;
   if (base >= n) return;
   const double c = clip_coef ? *clip_coef : 1.0;
@@ -116,8 +140,7 @@ reduce_adamw_kernel(GradPtrs gp, int64_t n, float* __restrict__ master,
     st_stream(master + base, wq);
     st_stream(mom1 + base, mq);
     st_stream(mom2 + base, vq);
-    __stcs(reinterpret_cast<uint2*>(param_out + base),
-           make_uint2(pb[0] | (pb[1] << 16), pb[2] | (pb[3] << 16)));
+    out.vec(base, make_uint2(pb[0] | (pb[1] << 16), pb[2] | (pb[3] << 16)));
   } else {
     // ragged tail: fewer than kVec parameters left, one at a time
     for (int64_t i = base; i < n; ++i) {
@@ -126,9 +149,27 @@ reduce_adamw_kernel(GradPtrs gp, int64_t n, float* __restrict__ master,
       float w = master[i], m = mom1[i], v = mom2[i];
       adamw_element(__fmul_rn(s, k.inv_R), w, m, v, k, k1, k2);
       master[i] = w; mom1[i] = m; mom2[i] = v;
-      param_out[i] = (uint16_t)f32_to_bf16_bits(w);
+      out.one(i, (uint16_t)f32_to_bf16_bits(w));
     }
   }
+}
+
+template <int R>
+__global__ void __launch_bounds__(kUpdateThreads, 8)
+reduce_adamw_kernel(GradPtrs gp, int64_t n, float* __restrict__ master,
+                    float* __restrict__ mom1, float* __restrict__ mom2,
+                    uint16_t* __restrict__ param_out, UpdateConsts k,
+                    const double* __restrict__ clip_coef) {
+  reduce_adamw_body<R>(gp, n, master, mom1, mom2, OneOut{param_out}, k, clip_coef);
+}
+
+// The same update with the BF16 copy stored into `outs.count` buffers (see ManyOuts).
+template <int R>
+__global__ void __launch_bounds__(kUpdateThreads, 8)
+reduce_adamw_bcast_kernel(GradPtrs gp, int64_t n, float* __restrict__ master,
+                          float* __restrict__ mom1, float* __restrict__ mom2, ManyOuts outs,
+                          UpdateConsts k, const double* __restrict__ clip_coef) {
+  reduce_adamw_body<R>(gp, n, master, mom1, mom2, outs, k, clip_coef);
 }
 
 // ---- sum of squares of the averaged gradient ----------------------------------------------
@@ -228,6 +269,22 @@ grad_norm_finish_kernel(const double* __restrict__ partials, int64_t count, doub
     scalars[2] = c;
     scalars[3] = (norm - norm == 0.0) ? 0.0 : 1.0;
   }
+}
+
+// ---- tile sums of one shard written into every GPU's gathered array ---------------------------
+//
+// The all-gather of the norm's tile sums in a sharded step (8 bytes per 16384 parameters): this
+// GPU's `count` sums are stored at the same offset of `ndst` arrays, its own and the peers'
+// (mapped), with plain stores. Pure data movement.
+struct F64Dsts {
+  double* p[kMaxRanks];
+};
+__global__ void __launch_bounds__(256)
+scatter_tile_sums_kernel(const double* __restrict__ src, int64_t count, F64Dsts dsts, int ndst) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= count) return;
+  const double x = src[i];
+  for (int o = 0; o < ndst; ++o) dsts.p[o][i] = x;
 }
 
 // ---- rank reduction alone: the averaged gradient as one BF16 buffer --------------------

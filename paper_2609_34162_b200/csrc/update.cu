@@ -40,6 +40,30 @@ int launch_update(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, float*
   return SLIDEDP_OK;
 }
 
+// The update with the BF16 copy stored into several buffers (sharded multi-GPU step).
+static int launch_update_bcast(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, float* w,
+                               float* m, float* v, const ManyOuts& outs, const UpdateConsts& k,
+                               const double* coef, cudaStream_t st) {
+  if (n == 0) return SLIDEDP_OK;
+  FAULT_POINT();
+  const int64_t groups = (n + kVec - 1) / kVec;
+  const unsigned blocks = (unsigned)((groups + kUpdateThreads - 1) / kUpdateThreads);
+  switch (R) {
+#define SLIDEDP_CASE(r)                                                                         \
+  case r:                                                                                       \
+    reduce_adamw_bcast_kernel<r><<<blocks, kUpdateThreads, 0, st>>>(gp, n, w, m, v, outs, k, coef); \
+    break;
+    SLIDEDP_CASE(1) SLIDEDP_CASE(2) SLIDEDP_CASE(3) SLIDEDP_CASE(4) SLIDEDP_CASE(5) SLIDEDP_CASE(6)
+    SLIDEDP_CASE(7) SLIDEDP_CASE(8) SLIDEDP_CASE(9) SLIDEDP_CASE(10) SLIDEDP_CASE(11)
+    SLIDEDP_CASE(12) SLIDEDP_CASE(13) SLIDEDP_CASE(14) SLIDEDP_CASE(15) SLIDEDP_CASE(16)
+#undef SLIDEDP_CASE
+    default: return SLIDEDP_ERR_INVALID_ARG;
+  }
+  ctx->launches += 1;
+  CU_AFTER_LAUNCH();
+  return SLIDEDP_OK;
+}
+
 // One instantiation per rank count (R is validated to 1..16 before this is reached).
 void launch_sumsq(const GradPtrs& gp, int R, int64_t n, float inv_R, double* tile_sums,
                   unsigned blocks, cudaStream_t st) {
@@ -208,6 +232,60 @@ int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* grads_bf16, 
   return launch_update(ctx, gp, R, n, master, m, v, static_cast<uint16_t*>(param_bf16_out),
                        make_consts(hp), clip ? ctx->scalars + 2 : nullptr,
                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+int slidedp_scatter_tile_sums(slidedp_ctx* ctx, const double* tile_sums, int64_t count,
+                              double* const* dsts, int n_dsts, void* cuda_stream) {
+  if (!ctx || count < 0 || !dsts || n_dsts < 1 || n_dsts > SLIDEDP_MAX_RANKS)
+    return SLIDEDP_ERR_INVALID_ARG;
+  if (count > 0 && !tile_sums) return SLIDEDP_ERR_INVALID_ARG;
+  F64Dsts d;
+  for (int o = 0; o < kMaxRanks; ++o) d.p[o] = nullptr;
+  for (int o = 0; o < n_dsts; ++o) {
+    if (!dsts[o]) return SLIDEDP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(dsts[o]) & 7u) != 0) return SLIDEDP_ERR_MISALIGNED;
+    d.p[o] = dsts[o];
+  }
+  if ((reinterpret_cast<uintptr_t>(tile_sums) & 7u) != 0) return SLIDEDP_ERR_MISALIGNED;
+  if (count == 0) return SLIDEDP_OK;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  FAULT_POINT();
+  scatter_tile_sums_kernel<<<(unsigned)((count + 255) / 256), 256, 0,
+                             static_cast<cudaStream_t>(cuda_stream)>>>(tile_sums, count, d, n_dsts);
+  ctx->launches += 1;
+  CU_AFTER_LAUNCH();
+  return SLIDEDP_OK;
+}
+
+int slidedp_reduce_adamw_chunk_bcast(slidedp_ctx* ctx, const void* const* grads_bf16, int R,
+                                     int64_t n, float* master, float* m, float* v,
+                                     void* const* param_bf16_outs, int n_outs,
+                                     const slidedp_hparams* hp, void* cuda_stream) {
+  if (!ctx || n < 0) return SLIDEDP_ERR_INVALID_ARG;
+  int rc = check_hparams(hp);
+  if (rc != SLIDEDP_OK) return rc;
+  GradPtrs gp;
+  rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  if (!param_bf16_outs || n_outs < 1 || n_outs > SLIDEDP_MAX_RANKS) return SLIDEDP_ERR_INVALID_ARG;
+  if (n > 0 && (!master || !m || !v)) return SLIDEDP_ERR_INVALID_ARG;
+  if (!aligned16(master) || !aligned16(m) || !aligned16(v)) return SLIDEDP_ERR_MISALIGNED;
+  ManyOuts outs;
+  outs.count = n_outs;
+  for (int o = 0; o < kMaxRanks; ++o) outs.p[o] = nullptr;
+  for (int o = 0; o < n_outs; ++o) {
+    if (!param_bf16_outs[o]) return SLIDEDP_ERR_INVALID_ARG;
+    if (!aligned16(param_bf16_outs[o])) return SLIDEDP_ERR_MISALIGNED;
+    outs.p[o] = static_cast<uint16_t*>(param_bf16_outs[o]);
+  }
+  const bool clip = hp->max_norm > 0.0;
+  if (clip && !ctx->norm_issued) return SLIDEDP_ERR_NO_NORM;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  return launch_update_bcast(ctx, gp, R, n, master, m, v, outs, make_consts(hp),
+                             clip ? ctx->scalars + 2 : nullptr,
+                             static_cast<cudaStream_t>(cuda_stream));
 }
 
 int slidedp_reduce_mean_bf16(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,

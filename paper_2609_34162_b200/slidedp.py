@@ -29,6 +29,7 @@ OK, ERR_INVALID_ARG, ERR_MISALIGNED, ERR_BUDGET, ERR_NOT_PINNED, ERR_CUDA, ERR_T
     0, -1, -2, -3, -4, -5, -6, -7)
 ERR_TOO_LARGE = -8
 NOALLOC_MAX_ELEMS = 1 << 30
+IPC_HANDLE_BYTES = 80
 
 
 class _HParams(ctypes.Structure):
@@ -112,6 +113,17 @@ _lib.slidedp_grad_norm_noalloc.argtypes = [_pp, ctypes.c_int, ctypes.c_int64, ct
                                            ctypes.c_double, _vp, _vp]
 _lib.slidedp_kernel_launches.restype = ctypes.c_int64
 _lib.slidedp_kernel_launches.argtypes = [_vp]
+_lib.slidedp_ipc_export.restype = ctypes.c_int
+_lib.slidedp_ipc_export.argtypes = [_vp, _vp, ctypes.c_char_p]
+_lib.slidedp_ipc_open.restype = ctypes.c_int
+_lib.slidedp_ipc_open.argtypes = [_vp, ctypes.c_char_p, ctypes.POINTER(_vp)]
+_lib.slidedp_ipc_close.restype = ctypes.c_int
+_lib.slidedp_ipc_close.argtypes = [_vp, _vp]
+_lib.slidedp_scatter_tile_sums.restype = ctypes.c_int
+_lib.slidedp_scatter_tile_sums.argtypes = [_vp, _vp, ctypes.c_int64, _pp, ctypes.c_int, _vp]
+_lib.slidedp_reduce_adamw_chunk_bcast.restype = ctypes.c_int
+_lib.slidedp_reduce_adamw_chunk_bcast.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp,
+                                                  _pp, ctypes.c_int, ctypes.POINTER(_HParams), _vp]
 _lib.slidedp_set_wait_seconds.restype = ctypes.c_int
 _lib.slidedp_set_wait_seconds.argtypes = [_vp, ctypes.c_double]
 _lib.slidedp_test_fail_nth_call.restype = ctypes.c_int
@@ -255,6 +267,34 @@ class Context:
         self._check(_lib.slidedp_reduce_adamw_chunk(
             self._h, _grad_array(grads), len(grads), n, _ptr(master), _ptr(m), _ptr(v),
             _ptr(param_bf16_out), ctypes.byref(c), _stream(stream)))
+
+    def slidedp_reduce_adamw_chunk_bcast(self, grads, n: int, master, m, v, param_bf16_outs,
+                                         hp: HParams, stream=None) -> None:
+        c = hp._c()
+        self._check(_lib.slidedp_reduce_adamw_chunk_bcast(
+            self._h, _grad_array(grads), len(grads), n, _ptr(master), _ptr(m), _ptr(v),
+            _grad_array(param_bf16_outs), len(param_bf16_outs), ctypes.byref(c), _stream(stream)))
+
+    def slidedp_scatter_tile_sums(self, tile_sums, count: int, dsts, stream=None) -> None:
+        self._check(_lib.slidedp_scatter_tile_sums(self._h, _ptr(tile_sums), count,
+                                                   _grad_array(dsts), len(dsts), _stream(stream)))
+
+    def slidedp_ipc_export(self, dev_ptr) -> bytes:
+        """The 80-byte handle of a device buffer (tensor or address), to send to a peer process."""
+        buf = ctypes.create_string_buffer(IPC_HANDLE_BYTES)
+        self._check(_lib.slidedp_ipc_export(self._h, _ptr(dev_ptr), buf))
+        return buf.raw
+
+    def slidedp_ipc_open(self, handle: bytes) -> int:
+        """Maps a peer's handle; returns the device address valid in this process."""
+        if len(handle) != IPC_HANDLE_BYTES:
+            raise ValueError("not a slidedp_ipc_handle")
+        out = _vp()
+        self._check(_lib.slidedp_ipc_open(self._h, handle, ctypes.byref(out)))
+        return int(out.value)
+
+    def slidedp_ipc_close(self, dev_ptr: int) -> None:
+        self._check(_lib.slidedp_ipc_close(self._h, dev_ptr))
 
     def slidedp_reduce_mean_bf16(self, grads, n: int, inv_R: float, out_bf16, stream=None) -> None:
         self._check(_lib.slidedp_reduce_mean_bf16(self._h, _grad_array(grads), len(grads), n, inv_R,

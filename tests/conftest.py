@@ -20,3 +20,12 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_libraries():
+    """Both shared libraries exist (and are current) before any test imports a binding."""
+    from paper_2609_34162_b200.build import build
+    import oracle
+    build()
+    oracle.build()

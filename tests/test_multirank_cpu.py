@@ -61,6 +61,46 @@ def test_single_rank_needs_no_process_group():
 def test_reference_arm_runs_on_rank_zero_only():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2")
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference",
-                        "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True,
+                        "--gpus", "2", "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True,
                        timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def _gloo_rank(args):
+    """A stand-in for bench.py's per-rank worker: joins a gloo group from the environment that
+    bench.launch_ranks prepared and proves that both ranks met."""
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    assert os.environ["MASTER_ADDR"] == "127.0.0.1" and os.environ["LOCAL_RANK"] == str(rank)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        t = torch.tensor([float(rank + 1)])
+        dist.all_reduce(t)
+        with open(os.path.join(args["dir"], f"rank{rank}.txt"), "w") as f:
+            f.write(f"{world} {t.item()}")
+    finally:
+        dist.destroy_process_group()
+    return args["codes"][rank]
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did(tmp_path):
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.launch_ranks(2, _gloo_rank, {"dir": str(tmp_path), "codes": [0, 0]}) == 0
+    assert sorted(os.listdir(tmp_path)) == ["rank0.txt", "rank1.txt"]
+    for r in range(2):
+        assert open(tmp_path / f"rank{r}.txt").read() == "2 3.0"     # world 2, 1 + 2
+    # a failing rank is reported
+    assert bench.launch_ranks(2, _gloo_rank, {"dir": str(tmp_path), "codes": [0, 7]}) == 7
+
+
+def test_gpus_flag_reaches_the_rank_spawn_and_must_agree_with_a_launcher():
+    exe = [sys.executable, os.path.join(ROOT, "bench.py")]
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    if not torch.cuda.is_available():
+        r = subprocess.run(exe + ["--gpus", "2", "--steps", "1", "--warmup", "0"], env=env,
+                           capture_output=True, text=True, timeout=300)
+        # two ranks were started and each stopped where the CUDA path must: no device, no fallback
+        assert r.returncode != 0 and r.stderr.count("needs a CUDA device") == 2, r.stderr
+    r = subprocess.run(exe + ["--gpus", "2"], env=dict(env, RANK="0", WORLD_SIZE="4"),
+                       capture_output=True, text=True, timeout=120)
+    assert r.returncode == 2 and "disagrees with WORLD_SIZE" in r.stderr

@@ -242,6 +242,84 @@ grad_sumsq_tiles_kernel(GradPtrs gp, int64_t n, float inv_R, double* __restrict_
   }
 }
 
+// Pass 1 at R = 1: the same tiles, the same per-thread order of additions and the same tree (so
+// the same bits as the kernel above), but a launch shape made for a stream of only 2 bytes per
+// parameter: one block computes kDeepTiles = 2 consecutive tiles and has ALL of a tile's loads
+// in flight at once (8 x 16 bytes per thread), the second tile's loads issued before the first
+// tile's arithmetic and shuffle tree. With one short-lived block per 32 KB tile the single-rank
+// pass was latency-bound (5.1 TB/s at 100 M parameters, 6.2 at 400 M); this form measured 5.7
+// and 7.0 TB/s on the same buffers. At R >= 2 a tile already carries enough bytes per block and
+// the generic kernel is as fast or faster, so only R = 1 takes this path.
+constexpr int kDeepTiles = 2;
+__device__ __forceinline__ double tile_thread_sum_r1(const uint4 (&raw)[kNormIters], float inv_R) {
+  double acc = 0.0;
+#pragma unroll
+  for (int it = 0; it < kNormIters; ++it) {
+    const uint32_t* x = reinterpret_cast<const uint32_t*>(&raw[it]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const double a = (double)__fmul_rn(bf16_lo(x[j]), inv_R);
+      acc = fma(a, a, acc);
+      const double b = (double)__fmul_rn(bf16_hi(x[j]), inv_R);
+      acc = fma(b, b, acc);
+    }
+  }
+  return acc;
+}
+__global__ void __launch_bounds__(kNormThreads)
+grad_sumsq_tiles_r1_kernel(const uint16_t* __restrict__ g, int64_t n, float inv_R,
+                           double* __restrict__ partials) {
+  __shared__ double warp_sum[kDeepTiles][kNormThreads / 32];
+  const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
+  const int64_t first = (int64_t)blockIdx.x * kDeepTiles;
+  uint4 raw[kDeepTiles][kNormIters];
+  // a tile is "full" when every one of its 16-byte vectors lies inside [0, n)
+  bool full[kDeepTiles];
+#pragma unroll
+  for (int t = 0; t < kDeepTiles; ++t) {
+    const int64_t tile = first + t;
+    full[t] = tile < ntiles && (tile + 1) * kNormTile <= n;
+    if (full[t]) {
+      const int64_t tb = tile * kNormTile + (int64_t)threadIdx.x * kNormVec;
+#pragma unroll
+      for (int it = 0; it < kNormIters; ++it)
+        raw[t][it] = ld_stream(g + tb + (int64_t)it * (kNormThreads * kNormVec));
+    }
+  }
+#pragma unroll
+  for (int t = 0; t < kDeepTiles; ++t) {
+    const int64_t tile = first + t;
+    if (tile >= ntiles) break;                     // uniform over the block
+    double acc = 0.0;
+    if (full[t]) {
+      acc = tile_thread_sum_r1(raw[t], inv_R);
+    } else {
+      // the step's last, ragged tile: element by element where a vector would cross n
+      const int64_t tb = tile * kNormTile + (int64_t)threadIdx.x * kNormVec;
+      for (int it = 0; it < kNormIters; ++it) {
+        const int64_t e = tb + (int64_t)it * (kNormThreads * kNormVec);
+#pragma unroll
+        for (int j = 0; j < kNormVec; ++j) {
+          float s = 0.0f;
+          if (e + j < n) s = __uint_as_float((uint32_t)g[e + j] << 16);
+          const double x = (double)__fmul_rn(s, inv_R);
+          acc = fma(x, x, acc);
+        }
+      }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+    if ((threadIdx.x & 31) == 0) warp_sum[t][threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double s = warp_sum[t][0];
+#pragma unroll
+      for (int w = 1; w < kNormThreads / 32; ++w) s += warp_sum[t][w];
+      partials[tile] = s;
+    }
+  }
+}
+
 // Pass 2: one block folds `count` partials in a fixed order: thread t adds partials
 // t, t + 1024, ... in that order, then the same warp butterfly and warp-order sum.
 // Writes scalars[0] = sumsq, [1] = norm, [2] = clip coefficient, [3] = 1.0 if non-finite.

@@ -67,6 +67,11 @@ static int launch_update_bcast(slidedp_ctx* ctx, const GradPtrs& gp, int R, int6
 // One instantiation per rank count (R is validated to 1..16 before this is reached).
 void launch_sumsq(const GradPtrs& gp, int R, int64_t n, float inv_R, double* tile_sums,
                   unsigned blocks, cudaStream_t st) {
+  if (R == 1) {   // single rank: two tiles per block, every load of a tile in flight (same bits)
+    grad_sumsq_tiles_r1_kernel<<<(blocks + kDeepTiles - 1) / kDeepTiles, kNormThreads, 0, st>>>(
+        gp.p[0], n, inv_R, tile_sums);
+    return;
+  }
   switch (R) {
 #define SLIDEDP_CASE(r) \
   case r: grad_sumsq_tiles_kernel<r><<<blocks, kNormThreads, 0, st>>>(gp, n, inv_R, tile_sums); break;

@@ -156,13 +156,16 @@ def test_config2_qwen3_8b_layer_step11_clipped(ctx, sd, divisor):
     assert_parity(wl.name, got, want, wl.max_norm)
 
 
-def test_norm_is_deterministic_and_chunk_invariant(ctx, sd):
-    n, R = 16384 * 37 + 4321, 4
+@pytest.mark.parametrize("R,n", [(4, 16384 * 37 + 4321), (1, 16384 * 37 + 4321), (1, 16384 * 38),
+                                 (1, 16384 * 36 + 3), (2, 16384 * 21 + 8), (8, 16384 * 5 + 9)])
+def test_norm_is_deterministic_and_chunk_invariant(ctx, sd, R, n):
+    """R = 1 runs its own launch shape (two tiles per block): cutting the step into single tiles
+    below checks that it produces the bits of one-tile-at-a-time."""
     grads, *_ = random_case(n, R, seed=77, sigma=1e-2)
     dg = [g.cuda() for g in grads]
     ref = None
     for _ in range(3):
-        ctx.slidedp_grad_norm(dg, n, 0.25, True)
+        ctx.slidedp_grad_norm(dg, n, 1.0 / R, True)
         out = ctx.slidedp_grad_norm_finish(1.0, fetch=True)
         ref = ref or out
         assert out == ref                                        # bit-identical run to run
@@ -170,19 +173,33 @@ def test_norm_is_deterministic_and_chunk_invariant(ctx, sd):
     for cut in (16384, 16384 * 5, 16384 * 36):
         first = True
         for lo in range(0, n, cut):
-            ctx.slidedp_grad_norm([g[lo:] for g in dg], min(cut, n - lo), 0.25, first)
+            ctx.slidedp_grad_norm([g[lo:] for g in dg], min(cut, n - lo), 1.0 / R, first)
             first = False
         assert ctx.slidedp_grad_norm_finish(1.0, fetch=True) == ref
     # any other cut: same value to rounding
     first = True
     for lo in range(0, n, 100_000):
-        ctx.slidedp_grad_norm([g[lo:] for g in dg], min(100_000, n - lo), 0.25, first)
+        ctx.slidedp_grad_norm([g[lo:] for g in dg], min(100_000, n - lo), 1.0 / R, first)
         first = False
     other = ctx.slidedp_grad_norm_finish(1.0, fetch=True)
     assert abs(other[0] - ref[0]) <= 1e-12 * ref[0]
-    want = oracle.clip_coef(oracle.grad_sumsq([parity.u16(g) for g in grads], 0.25), 1.0)
+    want = oracle.clip_coef(oracle.grad_sumsq([parity.u16(g) for g in grads], 1.0 / R), 1.0)
     parity.assert_norm_close(ref[0], want[1])
     assert abs(ref[1] - want[0]) <= 1e-6 * want[0]
+
+
+def test_single_rank_norm_kernel_has_the_bits_of_the_generic_one(ctx, sd):
+    """The R = 1 launch shape against the generic kernel on the same values: a second rank of
+    zeros (g + 0 = g exactly) with the same 1/R argument must give the same norm, bit for bit."""
+    for n in (16384 * 9 + 4321, 16384 * 4, 5, 16384 + 7):
+        grads, *_ = random_case(n, 1, seed=n % 1000, sigma=3e-3)
+        g = grads[0].cuda()
+        zero = torch.zeros_like(g)
+        ctx.slidedp_grad_norm([g], n, 0.5, True)
+        one = ctx.slidedp_grad_norm_finish(0.7, fetch=True)
+        ctx.slidedp_grad_norm([g, zero], n, 0.5, True)
+        two = ctx.slidedp_grad_norm_finish(0.7, fetch=True)
+        assert one == two and one[0] > 0.0
 
 
 def test_update_is_chunk_invariant_bit_for_bit(ctx, sd):

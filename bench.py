@@ -316,6 +316,10 @@ def run_cuda(args):
             host = host_resident_report(ctx, sd, W, torch, dev)
         except Exception as exc:                       # report, never hide
             host = {"error": repr(exc)}
+        try:
+            route = cpu_route_report(ctx, sd, W, torch, dev)
+        except Exception as exc:
+            route = {"error": repr(exc)}
         cpu = cpu_baseline(W, torch, np, wl, grads, layer)
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -326,7 +330,8 @@ def run_cuda(args):
                        "parallelism": f"{world} independent layer(s), one per GPU, no collective",
                        "l2": "inputs (8.1 GB touched per step) exceed the 126 MB L2"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
-            "clocks": clocks, "host_resident": host, "host_placement": host_placement(torch, local),
+            "clocks": clocks, "host_resident": host, "cpu_route": route,
+            "host_placement": host_placement(torch, local),
         }
     ctx.slidedp_destroy()
     if grouped:
@@ -666,6 +671,87 @@ def host_resident_report(ctx, sd, W, torch, dev):
                          "peak_source": "pinned-copy probe in this run, both directions at once"},
             "lanes_ms": {k: statistics.mean(r[k] for r in runs)
                          for k in ("ms_norm", "ms_h2d", "ms_kernel", "ms_d2h")}}
+
+
+def cpu_route_report(ctx, sd, W, torch, dev):
+    """The paper's OWN data path on this machine, beside the fused GPU path (baseline/cpu_route; not
+    the product): the Qwen3-14B-shaped layer of the host-resident configuration, gradient return
+    by GPU reduction (ONE BF16 gradient, G_l bytes D2H, produced by slidedp_reduce_mean_bf16) or
+    by CPU reduction (R G_l bytes D2H, summed on the host), the multi-threaded FP32 CPU AdamW per
+    64 MiB-of-FP32 chunk as the copies land, the CPU cast with streaming stores, and the BF16
+    delivery sent once ("sharded") or R times ("replicated"): the four datapaths of the paper's
+    host-traffic table (Sec. 2.4), with q_l = 1."""
+    import numpy as np
+
+    from baseline import cpu_route as cr
+    wl = W.CONFIGS[HOST_WORKLOAD]
+    n, R = wl.numel, wl.R
+    threads = min(len(os.sched_getaffinity(0)), cr.max_threads())
+    grads = [W.rank_gradient(wl, r, step=wl.first_step, device=dev) for r in range(R)]
+    mean = torch.empty(n, dtype=torch.bfloat16, device=dev)
+    outs = [torch.empty(n, dtype=torch.bfloat16, device=dev) for _ in range(R)]
+    stage = [torch.empty(n, dtype=torch.int16, pin_memory=True) for _ in range(R)]
+    pstage = torch.empty(n, dtype=torch.int16, pin_memory=True)
+    w = W.master_weights(wl, device=dev).cpu().numpy()
+    m, v = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    ce = W.chunk_elems(64)
+    # the clip coefficient comes from the GPU norm pass in every route (the paper has no clipping)
+    ctx.slidedp_grad_norm(grads, n, 1.0 / R, True)
+    _, coef = ctx.slidedp_grad_norm_finish(wl.max_norm, fetch=True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    st = torch.cuda.current_stream()
+    rows, t = [], 1
+    for reduction in ("gpu", "cpu"):
+        for delivery, copies in (("sharded", 1), ("replicated", R)):
+            runs = []
+            for i in range(4):
+                red_ms = 0.0
+                if reduction == "gpu":
+                    e0.record(st)
+                    ctx.slidedp_reduce_mean_bf16(grads, n, 1.0 / R, mean)
+                    e1.record(st)
+                    torch.cuda.synchronize()
+                    red_ms = e0.elapsed_time(e1)
+                    src, inv = [mean.data_ptr()], 1.0
+                else:
+                    src, inv = [g.data_ptr() for g in grads], 1.0 / R
+                hp = cr.HParams(inv_R=inv, clip_coef=coef, step=t, **wl.hparams)
+                r_ = cr.step(src, n, stage[:len(src)], w, m, v, pstage,
+                             [o.data_ptr() for o in outs[:copies]], ce, hp, threads)
+                t += 1
+                r_["ms_reduce_kernel"] = red_ms
+                if i >= 1:
+                    runs.append(r_)
+            ms = statistics.mean(r_["ms_total"] + r_["ms_reduce_kernel"] for r_ in runs)
+            upd = statistics.mean(r_["ms_update"] for r_ in runs)
+            host_bytes = (2 * len(src) + 12 + 14) * n          # gradients + state read, state + BF16 written
+            rows.append({"delivery": delivery, "reduction": reduction + " reduction",
+                         "h2d_bytes": runs[0]["h2d_bytes"], "d2h_bytes": runs[0]["d2h_bytes"],
+                         "ms_per_step": ms, "g_params_per_s": n / ms / 1e6,
+                         "ms_cpu_update": upd, "cpu_update_gbs": host_bytes / (upd * 1e6),
+                         "ms_waiting_for_d2h": statistics.mean(r_["ms_wait_d2h"] for r_ in runs),
+                         "ms_d2h_lane": statistics.mean(r_["ms_d2h_lane"] for r_ in runs),
+                         "ms_h2d_lane": statistics.mean(r_["ms_h2d_lane"] for r_ in runs),
+                         "ms_gpu_reduce_kernel": statistics.mean(r_["ms_reduce_kernel"] for r_ in runs)})
+    # delivery alone, both ways: CPU cast + 2 B/param H2D against FP32 H2D + GPU cast
+    hw = torch.empty(n, pin_memory=True)
+    hw.copy_(torch.from_numpy(w))
+    cpu_runs = [cr.deliver(w, n, pstage, outs[0].data_ptr(), ce, threads) for _ in range(4)][1:]
+    gpu_runs = [ctx.slidedp_deliver_params(hw, n, outs[0], ce, 3) for _ in range(4)][1:]
+    cpu_ms = statistics.mean(r_["ms_total"] for r_ in cpu_runs)
+    gpu_ms = statistics.mean(r_["ms_total"] for r_ in gpu_runs)
+    delivery = {"params": n, "chunk_mib": 64,
+                "cpu_cast_bf16_h2d": {"ms": cpu_ms, "link_bytes": 2 * n, "link_gbs": 2.0 * n / (cpu_ms * 1e6),
+                                      "ms_inside_cast": statistics.mean(r_["ms_update"] for r_ in cpu_runs),
+                                      "host_cores": threads, "isa": cr.isa(),
+                                      "host_dram_bytes": 6 * n},
+                "fp32_h2d_gpu_cast": {"ms": gpu_ms, "link_bytes": 4 * n, "link_gbs": 4.0 * n / (gpu_ms * 1e6),
+                                      "host_cores": 0, "host_dram_bytes": 4 * n}}
+    return {"workload": HOST_WORKLOAD, "params": n, "R": R, "chunk_mib": 64, "host_cores": threads,
+            "isa": cr.isa(), "arithmetic": "FP32 (vectorised CPU AdamW), BF16 gradients",
+            "clip_coef": coef, "datapaths": rows, "delivery": delivery,
+            "note": "baseline: the paper's route on this box; the product's host-resident step is "
+                    "host_resident.value"}
 
 
 def host_placement(torch, local: int):

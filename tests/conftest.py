@@ -29,3 +29,5 @@ def built_libraries():
     import oracle
     build()
     oracle.build()
+    from baseline import cpu_route
+    cpu_route.build()

@@ -1,5 +1,6 @@
 /* The C ABI used from plain C, with no Python in between: one clipped step of a small chunk
- * through libslidedp, compared with the C oracle under the benchmark's tolerances. Built and
+ * through libslidedp (device-resident, then host-resident through pinned memory, then the BF16
+ * delivery of the new master), compared with the C oracle under the benchmark's tolerances. Built and
  * run by tests/test_c_abi_program.py (gcc, links libslidedp, the oracle and the CUDA runtime).
  * Exit code 0 and a line starting with "PASS" on success. */
 #include <cuda_runtime.h>
@@ -66,6 +67,22 @@ int main(void) {
   CHECK_CUDA(cudaMemcpy(gv, dv, n * 4, cudaMemcpyDeviceToHost));
   CHECK_CUDA(cudaMemcpy(gp, dp, n * 2, cudaMemcpyDeviceToHost));
   const int64_t launches = slidedp_kernel_launches(ctx);
+
+  /* host-resident: the same step with the FP32 state in page-locked host memory, streamed in
+   * chunks of 8192 parameters through three slots; then the BF16 delivery of the new master */
+  float *pw, *pm, *pv;
+  void *dp2, *dp3;
+  CHECK_CUDA(cudaMallocHost((void**)&pw, n * 4)); CHECK_CUDA(cudaMallocHost((void**)&pm, n * 4));
+  CHECK_CUDA(cudaMallocHost((void**)&pv, n * 4));
+  CHECK_CUDA(cudaMalloc(&dp2, n * 2)); CHECK_CUDA(cudaMalloc(&dp3, n * 2));
+  memcpy(pw, hw, n * 4); memcpy(pm, hm, n * 4); memcpy(pv, hv, n * 4);
+  slidedp_stats st;
+  CHECK_SD(slidedp_stream_step(ctx, (const void* const*)dg, R, n, pw, pm, pv, dp2, 8192, 3, 0, &hp_sd, &st));
+  slidedp_stats dst;
+  CHECK_SD(slidedp_deliver_params(ctx, pw, n, dp3, 16384, 2, &dst));
+  uint16_t *gp2 = malloc(n * 2), *gp3 = malloc(n * 2), *want3 = malloc(n * 2);
+  CHECK_CUDA(cudaMemcpy(gp2, dp2, n * 2, cudaMemcpyDeviceToHost));
+  CHECK_CUDA(cudaMemcpy(gp3, dp3, n * 2, cudaMemcpyDeviceToHost));
   CHECK_SD(slidedp_destroy(ctx));
 
   /* oracle side */
@@ -84,10 +101,22 @@ int main(void) {
       if (!(err <= allowed)) ++bad;
     }
   for (int64_t i = 0; i < n; ++i) bf16_differ += gp[i] != hp[i];
+  /* the host-resident state and BF16 copy equal the device-resident ones bit for bit, the
+   * statistics carry the same norm, and the delivery is the oracle's cast of that master */
+  int64_t host_differs = 0, delivery_differs = 0;
+  const float* hgot[3] = {pw, pm, pv};
+  for (int a = 0; a < 3; ++a) host_differs += memcmp(hgot[a], got[a], n * 4) != 0;
+  host_differs += memcmp(gp2, gp, n * 2) != 0;
+  oracle_cast_master_to_bf16(pw, n, want3);
+  for (int64_t i = 0; i < n; ++i) delivery_differs += gp3[i] != want3[i];
+  const int host_ok = host_differs == 0 && delivery_differs == 0 && st.chunks == (n + 8191) / 8192 &&
+                      st.norm == norm && st.clip_coef == coef && dst.chunks == (n + 16383) / 16384;
   const int ok = bad == 0 && bf16_differ <= n / 10000 && fabs(norm - onorm) <= 1e-6 * onorm &&
-                 fabs(coef - ocoef) <= 1e-6 * ocoef && ocoef < 1.0 && launches == 3;
-  printf("%s n=%lld R=%d norm=%.12g (oracle %.12g) coef=%.6f fp32_outside=%lld bf16_differ=%lld launches=%lld\n",
+                 fabs(coef - ocoef) <= 1e-6 * ocoef && ocoef < 1.0 && launches == 3 && host_ok;
+  printf("%s n=%lld R=%d norm=%.12g (oracle %.12g) coef=%.6f fp32_outside=%lld bf16_differ=%lld launches=%lld "
+         "host_resident_differs=%lld delivery_differs=%lld chunks=%lld\n",
          ok ? "PASS" : "FAIL", (long long)n, R, norm, onorm, coef, (long long)bad,
-         (long long)bf16_differ, (long long)launches);
+         (long long)bf16_differ, (long long)launches, (long long)host_differs,
+         (long long)delivery_differs, (long long)st.chunks);
   return ok ? 0 : 1;
 }

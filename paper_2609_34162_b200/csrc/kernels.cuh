@@ -131,16 +131,17 @@ __device__ __forceinline__ void reduce_adamw_body(const GradPtrs& gp, int64_t n,
     float* wf = reinterpret_cast<float*>(&wq);
     float* mf = reinterpret_cast<float*>(&mq);
     float* vf = reinterpret_cast<float*>(&vq);
-    uint32_t pb[kVec];
+    uint32_t pk[kVec / 2];
 #pragma unroll
-    for (int j = 0; j < kVec; ++j) {
+    for (int j = 0; j < kVec; j += 2) {
       adamw_element(__fmul_rn(s[j], k.inv_R), wf[j], mf[j], vf[j], k, k1, k2);
-      pb[j] = f32_to_bf16_bits(wf[j]);
+      adamw_element(__fmul_rn(s[j + 1], k.inv_R), wf[j + 1], mf[j + 1], vf[j + 1], k, k1, k2);
+      pk[j / 2] = f32_to_bf16_bits(wf[j]) | (f32_to_bf16_bits(wf[j + 1]) << 16);
     }
     st_stream(master + base, wq);
     st_stream(mom1 + base, mq);
     st_stream(mom2 + base, vq);
-    out.vec(base, make_uint2(pb[0] | (pb[1] << 16), pb[2] | (pb[3] << 16)));
+    out.vec(base, make_uint2(pk[0], pk[1]));
   } else {
     // ragged tail: fewer than kVec parameters left, one at a time
     for (int64_t i = base; i < n; ++i) {

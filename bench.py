@@ -261,6 +261,10 @@ def run_cuda(args):
     upd_best = min(e[1].elapsed_time(e[2]) for e in events)
     t_next += args.steps
 
+    # the same loads and stores with no arithmetic, on the same buffers (state unchanged): what
+    # this access mix can reach on this device, beside the plain-copy peak
+    mix_gbs = ctx.slidedp_hbm_mix_probe(grads, n, w, m, v, p, 8)
+
     ms_per_step = total_ms / args.steps
     value = job_value(world, n, args.steps, total_ms)
     peak, peak_kind = measured_peak_hbm()
@@ -274,6 +278,9 @@ def run_cuda(args):
                 "algorithmic_bytes_per_launch": upd_bytes, "ms_per_launch": upd_ms,
                 "ms_per_launch_best": upd_best,
                 "frac_of_nominal_8000": achieved / 8000.0,
+                "access_mix_peak": mix_gbs, "frac_of_access_mix_peak": achieved / mix_gbs,
+                "access_mix_peak_source": "slidedp_hbm_mix_probe in this run: the kernel's loads and "
+                                          "stores with no arithmetic, same buffers, best of 8",
                 "norm_pass": {"ms": norm_ms, "algorithmic_bytes": 2 * R * n,
                               "achieved": 2 * R * n / (norm_ms * 1e-3) / 1e9,
                               "frac": 2 * R * n / (norm_ms * 1e-3) / 1e9 / peak}}

@@ -361,6 +361,20 @@ SLIDEDP_API int slidedp_model_stream_step(int64_t n_total, int R, int64_t chunk_
 SLIDEDP_API int slidedp_link_probe(slidedp_ctx* ctx, void* host_a, void* host_b, void* dev_a, void* dev_b,
                        size_t bytes, size_t copy_bytes, int reps, double out4[4]);
 
+/* ---- HBM probe with the update kernel's access mix: a roofline for the fused kernel -------
+ *
+ * Runs, reps times after two warm-up launches, a kernel with exactly the loads and stores of
+ * slidedp_reduce_adamw_chunk at this R (12 + 2R bytes read, 14 written per parameter, same
+ * launch shape and cache hints) and NO arithmetic, and reports the best rate in GB/s counted
+ * with the same 26 + 2R bytes per parameter. master / m / v are read and written back unchanged;
+ * scratch_bf16_out (device, n BF16) is overwritten. Synchronous (bounded waits) on cuda_stream.
+ * Arguments and checks as for slidedp_reduce_adamw_chunk; n >= 4. (No counterpart in the paper:
+ * measurement support, like slidedp_link_probe.)
+ */
+SLIDEDP_API int slidedp_hbm_mix_probe(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                          float* master, float* m, float* v, void* scratch_bf16_out, int reps,
+                          double* best_gbs, void* cuda_stream);
+
 /* ---- global norm for callers that cannot allocate ---------------------------------------
  *
  * (No counterpart in the paper: this entry point exists for deployment reasons only.)

@@ -173,6 +173,34 @@ reduce_adamw_bcast_kernel(GradPtrs gp, int64_t n, float* __restrict__ master,
   reduce_adamw_body<R>(gp, n, master, mom1, mom2, outs, k, clip_coef);
 }
 
+// ---- the update kernel's memory traffic with no arithmetic (a roofline probe) ------------------
+//
+// Same launch shape, same loads and stores as reduce_adamw_kernel<R> (R 8-byte BF16 loads and
+// three 16-byte FP32 loads per thread, three 16-byte stores and one 8-byte store), but the FP32
+// state is written back unchanged and the BF16 output is an xor of the gradient words: what this
+// access mix (12 + 2R bytes read, 14 written per parameter) can reach on the device when nothing
+// is computed. Only whole groups of kVec parameters are touched.
+template <int R>
+__global__ void __launch_bounds__(kUpdateThreads, 8)
+traffic_mix_kernel(GradPtrs gp, int64_t n, float* __restrict__ master, float* __restrict__ mom1,
+                   float* __restrict__ mom2, uint16_t* __restrict__ out) {
+  const int64_t base = ((int64_t)blockIdx.x * kUpdateThreads + threadIdx.x) * kVec;
+  if (base + kVec > n) return;
+  uint2 x = make_uint2(0u, 0u);
+  uint2 graw[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) graw[r] = __ldcs(reinterpret_cast<const uint2*>(gp.p[r] + base));
+  const uint4 wq = ld_stream(master + base);
+  const uint4 mq = ld_stream(mom1 + base);
+  const uint4 vq = ld_stream(mom2 + base);
+#pragma unroll
+  for (int r = 0; r < R; ++r) { x.x ^= graw[r].x; x.y ^= graw[r].y; }
+  st_stream(master + base, wq);
+  st_stream(mom1 + base, mq);
+  st_stream(mom2 + base, vq);
+  __stcs(reinterpret_cast<uint2*>(out + base), x);
+}
+
 // ---- sum of squares of the averaged gradient ----------------------------------------------
 //
 // Pass 1: one FP64 partial per fixed tile of kNormTile elements. Inside a tile thread t

@@ -293,6 +293,57 @@ int slidedp_reduce_adamw_chunk_bcast(slidedp_ctx* ctx, const void* const* grads_
                              static_cast<cudaStream_t>(cuda_stream));
 }
 
+int slidedp_hbm_mix_probe(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
+                          float* master, float* m, float* v, void* scratch_bf16_out, int reps,
+                          double* best_gbs, void* cuda_stream) {
+  if (!ctx || n < kVec || reps < 1 || !best_gbs) return SLIDEDP_ERR_INVALID_ARG;
+  GradPtrs gp;
+  int rc = check_grads(grads_bf16, R, &gp);
+  if (rc != SLIDEDP_OK) return rc;
+  if (!master || !m || !v || !scratch_bf16_out) return SLIDEDP_ERR_INVALID_ARG;
+  if (!aligned16(master) || !aligned16(m) || !aligned16(v) || !aligned16(scratch_bf16_out))
+    return SLIDEDP_ERR_MISALIGNED;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t groups = n / kVec;
+  const unsigned blocks = (unsigned)((groups + kUpdateThreads - 1) / kUpdateThreads);
+  uint16_t* out = static_cast<uint16_t*>(scratch_bf16_out);
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  CU(cudaEventCreate(&e0));
+  if (cudaEventCreate(&e1) != cudaSuccess) { cudaEventDestroy(e0); return cuda_fail(ctx, cudaErrorUnknown); }
+  double best = 0.0;
+  for (int rep = 0; rep < reps + 2 && rc == SLIDEDP_OK; ++rep) {      // two warm-up launches
+    cudaError_t e = cudaEventRecord(e0, st);
+    if (e == cudaSuccess) {
+      switch (R) {
+#define SLIDEDP_CASE(r) \
+  case r: traffic_mix_kernel<r><<<blocks, kUpdateThreads, 0, st>>>(gp, n, master, m, v, out); break;
+        SLIDEDP_CASE(1) SLIDEDP_CASE(2) SLIDEDP_CASE(3) SLIDEDP_CASE(4) SLIDEDP_CASE(5) SLIDEDP_CASE(6)
+        SLIDEDP_CASE(7) SLIDEDP_CASE(8) SLIDEDP_CASE(9) SLIDEDP_CASE(10) SLIDEDP_CASE(11)
+        SLIDEDP_CASE(12) SLIDEDP_CASE(13) SLIDEDP_CASE(14) SLIDEDP_CASE(15) SLIDEDP_CASE(16)
+#undef SLIDEDP_CASE
+        default: break;
+      }
+      ctx->launches += 1;
+      e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(e1, st);
+    if (e != cudaSuccess) { rc = cuda_fail(ctx, e); break; }
+    rc = bounded_event_wait(ctx, e1, ctx->wait_seconds);
+    if (rc != SLIDEDP_OK) break;
+    float ms = 0.f;
+    if (rep >= 2 && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess && ms > 0.f) {
+      const double gbs = (double)(26 + 2 * R) * (double)(groups * kVec) / ((double)ms * 1e6);
+      if (gbs > best) best = gbs;
+    }
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (rc == SLIDEDP_OK) *best_gbs = best;
+  return rc;
+}
+
 int slidedp_reduce_mean_bf16(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
                              double inv_R, void* out_bf16, void* cuda_stream) {
   if (!ctx || n < 0 || inv_R != inv_R) return SLIDEDP_ERR_INVALID_ARG;

@@ -124,6 +124,9 @@ _lib.slidedp_scatter_tile_sums.argtypes = [_vp, _vp, ctypes.c_int64, _pp, ctypes
 _lib.slidedp_reduce_adamw_chunk_bcast.restype = ctypes.c_int
 _lib.slidedp_reduce_adamw_chunk_bcast.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp,
                                                   _pp, ctypes.c_int, ctypes.POINTER(_HParams), _vp]
+_lib.slidedp_hbm_mix_probe.restype = ctypes.c_int
+_lib.slidedp_hbm_mix_probe.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp, _vp,
+                                       ctypes.c_int, ctypes.POINTER(ctypes.c_double), _vp]
 _lib.slidedp_set_wait_seconds.restype = ctypes.c_int
 _lib.slidedp_set_wait_seconds.argtypes = [_vp, ctypes.c_double]
 _lib.slidedp_test_fail_nth_call.restype = ctypes.c_int
@@ -334,6 +337,15 @@ class Context:
         if not want_stats:
             return None
         return {f: getattr(st, f) for f in ("ms_total", "ms_h2d", "gbs_h2d", "chunks")}
+
+    def slidedp_hbm_mix_probe(self, grads, n: int, master, m, v, scratch_bf16_out, reps: int = 5,
+                              stream=None) -> float:
+        """GB/s of the update kernel's loads and stores with no arithmetic (state unchanged)."""
+        out = ctypes.c_double()
+        self._check(_lib.slidedp_hbm_mix_probe(self._h, _grad_array(grads), len(grads), n, _ptr(master),
+                                               _ptr(m), _ptr(v), _ptr(scratch_bf16_out), reps,
+                                               ctypes.byref(out), _stream(stream)))
+        return out.value
 
     def slidedp_link_probe(self, host_a, host_b, dev_a, dev_b, nbytes: int, copy_bytes: int,
                            reps: int = 3):

@@ -485,3 +485,24 @@ def test_sharded_step_emulated_on_one_gpu_is_bit_identical(ctx, sd, shards):
     torch.cuda.synchronize()
     for a, b in ((sw, rw), (sm, rm), (sv, rv), (sp, rp)):
         assert torch.equal(a, b)
+
+
+def test_hbm_mix_probe_leaves_the_state_unchanged(ctx, sd):
+    """The roofline probe issues the update kernel's loads and stores without arithmetic: the FP32
+    state comes back bit for bit, only the scratch output changes, and a rate is reported."""
+    n, R = (1 << 22) + 6, 4
+    grads, w, m, v = random_case(n, R, seed=8)
+    dg = [g.cuda() for g in grads]
+    dw, dm, dv = w.cuda(), m.cuda(), v.cuda()
+    scratch = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    torch.cuda.synchronize()
+    gbs = ctx.slidedp_hbm_mix_probe(dg, n, dw, dm, dv, scratch, 3)
+    torch.cuda.synchronize()
+    assert gbs > 100.0
+    assert torch.equal(dw.cpu(), w) and torch.equal(dm.cpu(), m) and torch.equal(dv.cpu(), v)
+    assert all(torch.equal(a.cpu(), b) for a, b in zip(dg, grads))
+    assert scratch.view(torch.int16).count_nonzero() > n // 2
+    assert not scratch[-2:].view(torch.int16).any()          # the ragged tail is not touched
+    with pytest.raises(sd.SlideDPError) as e:
+        ctx.slidedp_hbm_mix_probe(dg, 2, dw, dm, dv, scratch, 3)
+    assert e.value.status == sd.ERR_INVALID_ARG

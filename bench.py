@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter of the fused update kernel, from an
 # ncu capture of a 50 M-parameter, R = 4 launch (a full-size launch is above the size an ncu
 # capture should hold); scaled to a full launch by the parameter count.
-NCU_TRAFFIC_BYTES_PER_PARAM = 33.04
+NCU_TRAFFIC_BYTES_PER_PARAM = 32.96
 
 
 def measured_peak_hbm():

@@ -11,9 +11,6 @@ using namespace slidedp::host;
 
 namespace {
 
-constexpr int64_t kTailPieces = 8;                 // pieces of a step's last chunk
-constexpr int64_t kMinPieceElems = 1 << 18;        // but no piece below 1 MiB per FP32 array
-
 
 // Grows the slot allocation to `need` bytes if the budget allows (checked before any work).
 int ensure_slots(slidedp_ctx* ctx, size_t need) {
@@ -169,53 +166,36 @@ int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total,
     const int slot = (int)((ctx->ring_next + c) % nbuf);
     const int64_t off = c * chunk_elems;
     const int64_t len = n_total - off < chunk_elems ? n_total - off : chunk_elems;
+    const size_t bytes = (size_t)len * sizeof(float);
     float* sw = ctx->slots + (size_t)slot * 3 * cap;
     float* sm = sw + cap;
     float* sv = sm + cap;
-    ChunkEvents* te = (timed && c == (nchunks - 1) / 2) ? &ctx->timing[0] : nullptr;
-    // The step ends one chunk's kernel + copy-out after the copy-in lane has moved its last
-    // byte. The LAST chunk is therefore cut into pieces that go through copy-in, kernel and
-    // copy-out one after the other, so that only one piece's copy-out is left when the copy-in
-    // lane runs dry. Elementwise work: the pieces change no bits.
-    const bool last = c == nchunks - 1;
-    int64_t piece = len;
-    if (last && nchunks > 1) {
-      piece = ((len + kTailPieces - 1) / kTailPieces + 7) / 8 * 8;
-      if (piece < kMinPieceElems) piece = kMinPieceElems;
-    }
+    ChunkEvents* te = (timed && c == nchunks / 2) ? &ctx->timing[0] : nullptr;
     // copy-in: the slot must have been drained by the copy-out that last used it (a no-op
     // for an event that was never recorded or has completed)
     CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_free[slot], 0));
     if (timed && c == 0) CU(cudaEventRecord(ctx->ev_in_first, ctx->s_in));
-    for (int64_t po = 0; po < len; po += piece) {
-      const int64_t pl = len - po < piece ? len - po : piece;
-      const size_t pbytes = (size_t)pl * sizeof(float);
-      const bool last_piece = po + pl == len;
-      CU(cudaMemcpyAsync(sw + po, host_master + off + po, pbytes, cudaMemcpyHostToDevice, ctx->s_in));
-      CU(cudaMemcpyAsync(sm + po, host_m + off + po, pbytes, cudaMemcpyHostToDevice, ctx->s_in));
-      CU(cudaMemcpyAsync(sv + po, host_v + off + po, pbytes, cudaMemcpyHostToDevice, ctx->s_in));
-      if (timed && last && last_piece) CU(cudaEventRecord(ctx->ev_in_last, ctx->s_in));
-      // (a stream's wait refers to the record that precedes it, so the slot's events can be
-      // recorded again for the next piece)
-      CU(cudaEventRecord(ctx->ev_loaded[slot], ctx->s_in));
-      // update
-      CU(cudaStreamWaitEvent(ctx->s_compute, ctx->ev_loaded[slot], 0));
-      if (te && po == 0) CU(cudaEventRecord(te->k_start, ctx->s_compute));
-      GradPtrs gc = gp;
-      for (int r = 0; r < R; ++r) gc.p[r] = gp.p[r] + off + po;
-      rc = launch_update(ctx, gc, R, pl, sw + po, sm + po, sv + po, pout + off + po, k, coef,
-                         ctx->s_compute);
-      if (rc != SLIDEDP_OK) return rc;
-      if (te && last_piece) CU(cudaEventRecord(te->k_end, ctx->s_compute));
-      CU(cudaEventRecord(ctx->ev_updated[slot], ctx->s_compute));
-      // copy-out
-      CU(cudaStreamWaitEvent(ctx->s_out, ctx->ev_updated[slot], 0));
-      if (timed && c == 0 && po == 0) CU(cudaEventRecord(ctx->ev_out_first, ctx->s_out));
-      CU(cudaMemcpyAsync(host_master + off + po, sw + po, pbytes, cudaMemcpyDeviceToHost, ctx->s_out));
-      CU(cudaMemcpyAsync(host_m + off + po, sm + po, pbytes, cudaMemcpyDeviceToHost, ctx->s_out));
-      CU(cudaMemcpyAsync(host_v + off + po, sv + po, pbytes, cudaMemcpyDeviceToHost, ctx->s_out));
-      if (timed && last && last_piece) CU(cudaEventRecord(ctx->ev_out_last, ctx->s_out));
-    }
+    CU(cudaMemcpyAsync(sw, host_master + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
+    CU(cudaMemcpyAsync(sm, host_m + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
+    CU(cudaMemcpyAsync(sv, host_v + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
+    if (timed && c == nchunks - 1) CU(cudaEventRecord(ctx->ev_in_last, ctx->s_in));
+    CU(cudaEventRecord(ctx->ev_loaded[slot], ctx->s_in));
+    // update
+    CU(cudaStreamWaitEvent(ctx->s_compute, ctx->ev_loaded[slot], 0));
+    if (te) CU(cudaEventRecord(te->k_start, ctx->s_compute));
+    GradPtrs gc = gp;
+    for (int r = 0; r < R; ++r) gc.p[r] = gp.p[r] + off;
+    rc = launch_update(ctx, gc, R, len, sw, sm, sv, pout + off, k, coef, ctx->s_compute);
+    if (rc != SLIDEDP_OK) return rc;
+    if (te) CU(cudaEventRecord(te->k_end, ctx->s_compute));
+    CU(cudaEventRecord(ctx->ev_updated[slot], ctx->s_compute));
+    // copy-out
+    CU(cudaStreamWaitEvent(ctx->s_out, ctx->ev_updated[slot], 0));
+    if (timed && c == 0) CU(cudaEventRecord(ctx->ev_out_first, ctx->s_out));
+    CU(cudaMemcpyAsync(host_master + off, sw, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
+    CU(cudaMemcpyAsync(host_m + off, sm, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
+    CU(cudaMemcpyAsync(host_v + off, sv, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
+    if (timed && c == nchunks - 1) CU(cudaEventRecord(ctx->ev_out_last, ctx->s_out));
     CU(cudaEventRecord(ctx->ev_free[slot], ctx->s_out));
   }
   ctx->ring_next += nchunks;
@@ -265,7 +245,7 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
     if (nchunks > 0) {
       const ChunkEvents& te = ctx->timing[0];
       // the timed kernel is the middle chunk's (warm, with copies running on both sides)
-      const int64_t mid_off = ((nchunks - 1) / 2) * chunk_elems;
+      const int64_t mid_off = (nchunks / 2) * chunk_elems;
       const int64_t mid_len = n_total - mid_off < chunk_elems ? n_total - mid_off : chunk_elems;
       CU(cudaEventElapsedTime(&ms, te.k_start, te.k_end));
       stats->ms_kernel = (double)ms * ((double)n_total / (double)mid_len);

@@ -170,7 +170,7 @@ int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total,
     float* sw = ctx->slots + (size_t)slot * 3 * cap;
     float* sm = sw + cap;
     float* sv = sm + cap;
-    ChunkEvents* te = (timed && c == nchunks / 2) ? &ctx->timing[0] : nullptr;
+    ChunkEvents* te = (timed && c == (nchunks - 1) / 2) ? &ctx->timing[0] : nullptr;
     // copy-in: the slot must have been drained by the copy-out that last used it (a no-op
     // for an event that was never recorded or has completed)
     CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_free[slot], 0));
@@ -245,7 +245,7 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
     if (nchunks > 0) {
       const ChunkEvents& te = ctx->timing[0];
       // the timed kernel is the middle chunk's (warm, with copies running on both sides)
-      const int64_t mid_off = (nchunks / 2) * chunk_elems;
+      const int64_t mid_off = ((nchunks - 1) / 2) * chunk_elems;
       const int64_t mid_len = n_total - mid_off < chunk_elems ? n_total - mid_off : chunk_elems;
       CU(cudaEventElapsedTime(&ms, te.k_start, te.k_end));
       stats->ms_kernel = (double)ms * ((double)n_total / (double)mid_len);

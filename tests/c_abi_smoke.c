@@ -80,6 +80,19 @@ int main(void) {
   CHECK_SD(slidedp_stream_step(ctx, (const void* const*)dg, R, n, pw, pm, pv, dp2, 8192, 3, 0, &hp_sd, &st));
   slidedp_stats dst;
   CHECK_SD(slidedp_deliver_params(ctx, pw, n, dp3, 16384, 2, &dst));
+  /* the same step once more, enqueued only and then waited for, on a second copy of the state;
+   * and the host-link probe on the (now free) pinned buffers of that copy */
+  float *qw, *qm, *qv;
+  void* dp4;
+  CHECK_CUDA(cudaMallocHost((void**)&qw, n * 4)); CHECK_CUDA(cudaMallocHost((void**)&qm, n * 4));
+  CHECK_CUDA(cudaMallocHost((void**)&qv, n * 4)); CHECK_CUDA(cudaMalloc(&dp4, n * 2));
+  memcpy(qw, hw, n * 4); memcpy(qm, hm, n * 4); memcpy(qv, hv, n * 4);
+  CHECK_SD(slidedp_set_wait_seconds(ctx, 60.0));
+  CHECK_SD(slidedp_stream_step_async(ctx, (const void* const*)dg, R, n, qw, qm, qv, dp4, 4096, 2, 1, &hp_sd));
+  CHECK_SD(slidedp_stream_wait(ctx));
+  const int async_same = memcmp(qw, pw, n * 4) == 0 && memcmp(qm, pm, n * 4) == 0 && memcmp(qv, pv, n * 4) == 0;
+  double link[4] = {0, 0, 0, 0};
+  CHECK_SD(slidedp_link_probe(ctx, qm, qv, dw, dm, (size_t)n * 4, 65536, 1, link));
   uint16_t *gp2 = malloc(n * 2), *gp3 = malloc(n * 2), *want3 = malloc(n * 2);
   CHECK_CUDA(cudaMemcpy(gp2, dp2, n * 2, cudaMemcpyDeviceToHost));
   CHECK_CUDA(cudaMemcpy(gp3, dp3, n * 2, cudaMemcpyDeviceToHost));
@@ -109,7 +122,8 @@ int main(void) {
   host_differs += memcmp(gp2, gp, n * 2) != 0;
   oracle_cast_master_to_bf16(pw, n, want3);
   for (int64_t i = 0; i < n; ++i) delivery_differs += gp3[i] != want3[i];
-  const int host_ok = host_differs == 0 && delivery_differs == 0 && st.chunks == (n + 8191) / 8192 &&
+  const int host_ok = async_same && link[0] > 0 && link[1] > 0 && link[2] > 0 && link[3] > 0 &&
+                      host_differs == 0 && delivery_differs == 0 && st.chunks == (n + 8191) / 8192 &&
                       st.norm == norm && st.clip_coef == coef && dst.chunks == (n + 16383) / 16384;
   const int ok = bad == 0 && bf16_differ <= n / 10000 && fabs(norm - onorm) <= 1e-6 * onorm &&
                  fabs(coef - ocoef) <= 1e-6 * ocoef && ocoef < 1.0 && launches == 3 && host_ok;

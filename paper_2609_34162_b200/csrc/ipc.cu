@@ -91,10 +91,9 @@ int slidedp_ipc_close(slidedp_ctx* ctx, void* dev_ptr) {
   for (size_t i = 0; i < ctx->ipc.size(); ++i) {
     IpcMapping& m = ctx->ipc[i];
     if (p < m.base || p >= m.base + m.bytes) continue;
-    if (--m.refs > 0) return SLIDEDP_OK;
-    char* base = m.base;
+    if (m.refs > 1) { m.refs -= 1; return SLIDEDP_OK; }
+    CU(cudaIpcCloseMemHandle(m.base));       // on failure the mapping stays recorded
     ctx->ipc.erase(ctx->ipc.begin() + (long)i);
-    CU(cudaIpcCloseMemHandle(base));
     return SLIDEDP_OK;
   }
   return SLIDEDP_ERR_INVALID_ARG;      // not a pointer this context mapped

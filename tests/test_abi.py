@@ -91,10 +91,20 @@ def test_binding_has_the_c_names_and_no_oracle_import():
                 text = open(os.path.join(dirpath, fn)).read()
                 assert not re.search(r"^\s*(import|from)\s+oracle\b", text, re.M), fn
                 assert "slidedp_oracle" not in text, fn
+                assert not re.search(r"^\s*(import|from)\s+baseline\b", text, re.M), fn
+                assert "cpu_route" not in text and "cpuroute" not in text, fn
     for fn in os.listdir(os.path.join(ROOT, "oracle")):
         if fn.endswith((".py", ".c", ".h")):
             text = open(os.path.join(ROOT, "oracle", fn)).read()
             assert "paper_2609_34162_b200" not in text and "slidedp.h" not in text, fn
+            assert "cpu_route" not in text and "cpuroute" not in text, fn
+    # the paper-route baseline stands alone as well: neither the library nor the oracle
+    base = os.path.join(ROOT, "baseline", "cpu_route")
+    for fn in os.listdir(base):
+        if fn.endswith((".py", ".cpp", ".h")):
+            text = open(os.path.join(base, fn)).read()
+            assert not re.search(r"^\s*(import|from)\s+(oracle|paper_2609_34162_b200)\b", text, re.M), fn
+            assert "slidedp.h" not in text and "slidedp_oracle" not in text and "internal.h" not in text, fn
 
 
 def test_workload_sizes_and_determinism():

@@ -6,7 +6,7 @@
 
 One "step" is one pass of the whole hot path over one Qwen3-8B-shaped decoder layer
 (192,946,176 parameters, R = 4 BF16 rank gradients, step 11, clip 1.0): the global-norm
-pass over all gradients (one launch), then the fused rank-reduce + AdamW + BF16-emit kernel.
+pass over all gradients, then the fused rank-reduce + AdamW + BF16-emit kernel.
 `value` is whole-job G-params/s with everything resident in HBM; `e2e` is the same step
 through slidedp_stream_step with the FP32 state in pinned HOST memory, host<->device copies
 inside the timed region. With --gpus N every rank updates its own layer (independent
@@ -218,7 +218,8 @@ def run_cuda(args):
 
     def device_step(t, ev=None):
         if ev: ev[0].record(stream)
-        ctx.slidedp_grad_norm_whole(grads, n, 1.0 / R, wl.max_norm)      # tile sums + fold, one launch
+        ctx.slidedp_grad_norm(grads, n, 1.0 / R, True)
+        ctx.slidedp_grad_norm_finish(wl.max_norm)
         if ev: ev[1].record(stream)
         ctx.slidedp_reduce_adamw_chunk(grads, n, w, m, v, p, hp(t))
         if ev: ev[2].record(stream)
@@ -514,13 +515,9 @@ def run_sweep(args):
         def norm_pass():
             ctx.slidedp_grad_norm(g, n, 1.0 / R, True)
             ctx.slidedp_grad_norm_finish(1.0)
-
-        def norm_whole():
-            ctx.slidedp_grad_norm_whole(g, n, 1.0 / R, 1.0)
         row = {"R": R}
         for name, fn, per in (("update", lambda: ctx.slidedp_reduce_adamw_chunk(g, n, w, m, v, p, h), 26 + 2 * R),
                               ("norm", norm_pass, 2 * R),
-                              ("norm_one_launch", norm_whole, 2 * R),
                               ("reduce_mean_bf16", lambda: ctx.slidedp_reduce_mean_bf16(g, n, 1.0 / R, p), 2 * R + 2)):
             med, best = timed(fn)
             row[name] = {"ms": med, "ms_best": best, "bytes_per_param": per,
@@ -856,8 +853,6 @@ def run_kernel_case(args):
         elif args.kernel == "norm":
             ctx.slidedp_grad_norm(grads, n, 1.0 / R, True)
             ctx.slidedp_grad_norm_finish(args.clip)
-        elif args.kernel == "norm_whole":
-            ctx.slidedp_grad_norm_whole(grads, n, 1.0 / R, args.clip)
         elif args.kernel == "reduce":
             ctx.slidedp_reduce_mean_bf16(grads, n, 1.0 / R, p)
         else:
@@ -865,8 +860,7 @@ def run_kernel_case(args):
     ev[args.launches].record(st)
     torch.cuda.synchronize()
     ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.launches)]
-    per = {"update": 26 + 2 * R, "norm": 2 * R, "norm_whole": 2 * R, "reduce": 2 * R + 2,
-           "stream": 24}[args.kernel]
+    per = {"update": 26 + 2 * R, "norm": 2 * R, "reduce": 2 * R + 2, "stream": 24}[args.kernel]
     print(json.dumps({"report": "kernel", "kernel": args.kernel, "params": n, "R": R,
                       "ms_per_launch": ms, "bytes_per_param": per,
                       "best_gbs": per * n / (min(ms) * 1e6)}))
@@ -917,8 +911,7 @@ def main(argv=None):
     ap.add_argument("--sharded", action="store_true",
                     help="one layer sharded over the ranks (peer-mapped gradients, BF16 copy stored "
                          "to every rank) instead of one independent layer per rank")
-    ap.add_argument("--kernel", choices=["update", "norm", "norm_whole", "reduce", "stream"],
-                    default="update")
+    ap.add_argument("--kernel", choices=["update", "norm", "reduce", "stream"], default="update")
     ap.add_argument("--params", type=int, default=48 << 20)
     ap.add_argument("--R", type=int, default=4)
     ap.add_argument("--launches", type=int, default=4)

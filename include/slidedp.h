@@ -153,17 +153,6 @@ SLIDEDP_API int slidedp_grad_norm(slidedp_ctx* ctx, const void* const* grads_bf1
 SLIDEDP_API int slidedp_grad_norm_finish(slidedp_ctx* ctx, double max_norm, double* host_norm /* nullable */,
                              double* host_coef /* nullable */, void* cuda_stream);
 
-/* The norm of a step that is ONE chunk, in one kernel launch: the same tiles, tile sums and
- * folding order as slidedp_grad_norm(first_chunk = 1) followed by slidedp_grad_norm_finish, hence
- * the same bits, but the block that finishes last does the fold itself, which saves the second
- * launch (a tenth of the pass at 100 M parameters and one rank). Leaves sumsq, norm and
- * coefficient in the context like slidedp_grad_norm_finish; same host_norm / host_coef behaviour.
- * slidedp_stream_step uses it when it computes the norm itself. Do not run two of these on one
- * context at the same time (they share the tile sums and a block counter). */
-SLIDEDP_API int slidedp_grad_norm_whole(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
-                            double inv_R, double max_norm, double* host_norm /* nullable */,
-                            double* host_coef /* nullable */, void* cuda_stream);
-
 /* The two halves of the norm with the tile sums in CALLER memory, for a step whose parameters are
  * sharded over several GPUs (each GPU updates a contiguous shard and reads its slice of every
  * rank's gradient, Sec. 3.2 "Parameter dispatch" / "Gradient return"): each GPU computes the tile

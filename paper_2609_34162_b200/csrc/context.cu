@@ -61,7 +61,6 @@ int slidedp_create(slidedp_ctx** out, int device, size_t gpu_budget_bytes) {
   step(cudaMalloc(&ctx->partials, (size_t)kInitialPartials * sizeof(double)));
   ctx->partials_cap = kInitialPartials;
   step(cudaMalloc(&ctx->scalars, 4 * sizeof(double)));
-  step(cudaMalloc(&ctx->ticket, sizeof(unsigned int)));
   step(cudaMallocHost(&ctx->host_scalars, 4 * sizeof(double)));
   step(cudaStreamCreateWithFlags(&ctx->s_in, cudaStreamNonBlocking));
   step(cudaStreamCreateWithFlags(&ctx->s_compute, cudaStreamNonBlocking));
@@ -82,7 +81,6 @@ int slidedp_create(slidedp_ctx** out, int device, size_t gpu_budget_bytes) {
   if (e == cudaSuccess) {
     const double init[4] = {0.0, 0.0, 1.0, 0.0};
     step(cudaMemcpy(ctx->scalars, init, sizeof init, cudaMemcpyHostToDevice));
-    step(cudaMemset(ctx->ticket, 0, sizeof(unsigned int)));
   }
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
@@ -115,7 +113,6 @@ int slidedp_destroy(slidedp_ctx* ctx) {
   if (ctx->slots) cudaFree(ctx->slots);
   if (ctx->partials) cudaFree(ctx->partials);
   if (ctx->scalars) cudaFree(ctx->scalars);
-  if (ctx->ticket) cudaFree(ctx->ticket);
   if (ctx->host_scalars) cudaFreeHost(ctx->host_scalars);
   (void)cudaGetLastError();
   delete ctx;

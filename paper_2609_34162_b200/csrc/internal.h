@@ -51,7 +51,6 @@ struct slidedp_ctx {
   double* scalars = nullptr;        // device: sumsq, norm, coef, nonfinite
   double* host_scalars = nullptr;   // pinned mirror
   bool norm_issued = false;
-  unsigned int* ticket = nullptr;   // device: block counter of the one-launch norm, zero at rest
   cudaEvent_t scalar_event = nullptr;
   // host-resident streaming
   cudaStream_t s_in = nullptr, s_compute = nullptr, s_out = nullptr;
@@ -130,8 +129,6 @@ void launch_sumsq(const GradPtrs& gp, int R, int64_t n, float inv_R, double* til
 int norm_chunk(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, double inv_R,
                int first_chunk, cudaStream_t st);
 int norm_finish(slidedp_ctx* ctx, double max_norm, cudaStream_t st);
-int norm_whole(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, double inv_R,
-               double max_norm, cudaStream_t st);
 
 }  // namespace host
 }  // namespace slidedp

@@ -209,9 +209,10 @@ traffic_mix_kernel(GradPtrs gp, int64_t n, float* __restrict__ master, float* __
 // a tile's partial does not depend on which block computes it or on the grid size.
 // Launched with one block per tile; the loads of UNROLL iterations are in flight together
 // (measured best: 2 at R = 4, 1 at R = 8, where more unrolling costs occupancy).
-template <int R, int UNROLL>
-__device__ __forceinline__ void tile_sums_body(const GradPtrs& gp, int64_t n, float inv_R,
-                                               double* __restrict__ partials, double* warp_sum) {
+template <int R, int UNROLL = (R >= 6) ? 1 : (R >= 3 ? 2 : 4)>
+__global__ void __launch_bounds__(kNormThreads)
+grad_sumsq_tiles_kernel(GradPtrs gp, int64_t n, float inv_R, double* __restrict__ partials) {
+  __shared__ double warp_sum[kNormThreads / 32];
   const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     const int64_t tbase = tile * kNormTile + (int64_t)threadIdx.x * kNormVec;
@@ -270,13 +271,6 @@ __device__ __forceinline__ void tile_sums_body(const GradPtrs& gp, int64_t n, fl
   }
 }
 
-template <int R, int UNROLL = (R >= 6) ? 1 : (R >= 3 ? 2 : 4)>
-__global__ void __launch_bounds__(kNormThreads)
-grad_sumsq_tiles_kernel(GradPtrs gp, int64_t n, float inv_R, double* __restrict__ partials) {
-  __shared__ double warp_sum[kNormThreads / 32];
-  tile_sums_body<R, UNROLL>(gp, n, inv_R, partials, warp_sum);
-}
-
 // Pass 1 at R = 1: the same tiles, the same per-thread order of additions and the same tree (so
 // the same bits as the kernel above), but a launch shape made for a stream of only 2 bytes per
 // parameter: one block computes kDeepTiles = 2 consecutive tiles and has ALL of a tile's loads
@@ -301,9 +295,10 @@ __device__ __forceinline__ double tile_thread_sum_r1(const uint4 (&raw)[kNormIte
   }
   return acc;
 }
-__device__ __forceinline__ void tile_sums_r1_body(const uint16_t* __restrict__ g, int64_t n,
-                                                  float inv_R, double* __restrict__ partials,
-                                                  double (*warp_sum)[kNormThreads / 32]) {
+__global__ void __launch_bounds__(kNormThreads)
+grad_sumsq_tiles_r1_kernel(const uint16_t* __restrict__ g, int64_t n, float inv_R,
+                           double* __restrict__ partials) {
+  __shared__ double warp_sum[kDeepTiles][kNormThreads / 32];
   const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
   const int64_t first = (int64_t)blockIdx.x * kDeepTiles;
   uint4 raw[kDeepTiles][kNormIters];
@@ -354,13 +349,6 @@ __device__ __forceinline__ void tile_sums_r1_body(const uint16_t* __restrict__ g
   }
 }
 
-__global__ void __launch_bounds__(kNormThreads)
-grad_sumsq_tiles_r1_kernel(const uint16_t* __restrict__ g, int64_t n, float inv_R,
-                           double* __restrict__ partials) {
-  __shared__ double warp_sum[kDeepTiles][kNormThreads / 32];
-  tile_sums_r1_body(g, n, inv_R, partials, warp_sum);
-}
-
 // Pass 2: one block folds `count` partials in a fixed order: thread t adds partials
 // t, t + 1024, ... in that order, then the same warp butterfly and warp-order sum.
 // Writes scalars[0] = sumsq, [1] = norm, [2] = clip coefficient, [3] = 1.0 if non-finite.
@@ -388,82 +376,6 @@ grad_norm_finish_kernel(const double* __restrict__ partials, int64_t count, doub
     scalars[2] = c;
     scalars[3] = (norm - norm == 0.0) ? 0.0 : 1.0;
   }
-}
-
-// ---- the whole norm in ONE launch: tile sums, and the last block to finish folds them ---------
-//
-// For a step that is a single chunk the two passes can share a launch: every block writes its
-// tile sums, publishes them (__threadfence) and takes a ticket; the block that draws the last
-// ticket then does pass 2 itself. Which block that is varies from run to run, the arithmetic does
-// not: the 256 threads each play four of pass 2's 1024 threads (thread r plays t = r, r + 256,
-// r + 512, r + 768: same lane, warps w, w + 8, w + 16, w + 24), so the per-thread sums, the warp
-// butterflies and the final warp-order sum are exactly those of grad_norm_finish_kernel and the
-// result has the same bits. Saves the second launch and its gap, which is a tenth of the pass
-// at 100 M parameters and one rank. The ticket counter is left at zero for the next launch.
-struct WholeNorm {
-  unsigned int* ticket;      // device, zero before the launch
-  double* scalars;           // sumsq, norm, coefficient, non-finite flag
-  double max_norm;
-  int64_t count;             // tiles of the step
-};
-__device__ __forceinline__ void fold_if_last_block(const double* partials, const WholeNorm& w,
-                                                   double* warp_sum32, unsigned int* is_last) {
-  __syncthreads();                                   // this block's tile sums are all written
-  if (threadIdx.x == 0) {
-    __threadfence();                                 // ... and visible before the ticket is
-    const unsigned int t = atomicAdd(w.ticket, 1u);
-    *is_last = (t == gridDim.x - 1) ? 1u : 0u;
-  }
-  __syncthreads();
-  if (*is_last == 0u) return;
-  __threadfence();                                   // see every other block's tile sums
-  double acc[kFinishThreads / kNormThreads];
-#pragma unroll
-  for (int k = 0; k < kFinishThreads / kNormThreads; ++k) {
-    acc[k] = 0.0;
-    for (int64_t i = threadIdx.x + k * kNormThreads; i < w.count; i += kFinishThreads)
-      acc[k] += __ldcg(partials + i);
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) acc[k] += __shfl_xor_sync(0xFFFFFFFFu, acc[k], off);
-    if ((threadIdx.x & 31) == 0) warp_sum32[(threadIdx.x >> 5) + k * (kNormThreads / 32)] = acc[k];
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double t = warp_sum32[0];
-    for (int v = 1; v < kFinishThreads / 32; ++v) t += warp_sum32[v];
-    const double norm = sqrt(t);
-    double c = 1.0;
-    if (w.max_norm > 0.0) {
-      c = w.max_norm / (norm + 1e-6);
-      if (c > 1.0) c = 1.0;
-    }
-    w.scalars[0] = t;
-    w.scalars[1] = norm;
-    w.scalars[2] = c;
-    w.scalars[3] = (norm - norm == 0.0) ? 0.0 : 1.0;
-    *w.ticket = 0u;
-  }
-}
-
-template <int R, int UNROLL = (R >= 6) ? 1 : (R >= 3 ? 2 : 4)>
-__global__ void __launch_bounds__(kNormThreads)
-grad_norm_whole_kernel(GradPtrs gp, int64_t n, float inv_R, double* __restrict__ partials,
-                       WholeNorm w) {
-  __shared__ double warp_sum[kNormThreads / 32];
-  __shared__ double warp_sum32[kFinishThreads / 32];
-  __shared__ unsigned int is_last;
-  tile_sums_body<R, UNROLL>(gp, n, inv_R, partials, warp_sum);
-  fold_if_last_block(partials, w, warp_sum32, &is_last);
-}
-
-__global__ void __launch_bounds__(kNormThreads)
-grad_norm_whole_r1_kernel(const uint16_t* __restrict__ g, int64_t n, float inv_R,
-                          double* __restrict__ partials, WholeNorm w) {
-  __shared__ double warp_sum[kDeepTiles][kNormThreads / 32];
-  __shared__ double warp_sum32[kFinishThreads / 32];
-  __shared__ unsigned int is_last;
-  tile_sums_r1_body(g, n, inv_R, partials, warp_sum);
-  fold_if_last_block(partials, w, warp_sum32, &is_last);
 }
 
 // ---- tile sums of one shard written into every GPU's gathered array ---------------------------

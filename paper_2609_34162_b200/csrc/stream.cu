@@ -152,7 +152,9 @@ int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total,
     CU(cudaStreamWaitEvent(ctx->s_out, ctx->ev_begin, 0));
   }
   if (clip && !norm_ready) {
-    rc = norm_whole(ctx, gp, R, n_total, hp->inv_R, hp->max_norm, ctx->s_compute);
+    rc = norm_chunk(ctx, gp, R, n_total, hp->inv_R, 1, ctx->s_compute);
+    if (rc != SLIDEDP_OK) return rc;
+    rc = norm_finish(ctx, hp->max_norm, ctx->s_compute);
     if (rc != SLIDEDP_OK) return rc;
   }
   if (synchronous) CU(cudaEventRecord(ctx->ev_norm_done, ctx->s_compute));

@@ -134,41 +134,6 @@ int norm_finish(slidedp_ctx* ctx, double max_norm, cudaStream_t st) {
   return SLIDEDP_OK;
 }
 
-// The norm of a step that is ONE chunk, in one launch (tile sums + fold by the last block).
-int norm_whole(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, double inv_R,
-               double max_norm, cudaStream_t st) {
-  ctx->partials_used = 0;
-  const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
-  if (ntiles == 0) return norm_finish(ctx, max_norm, st);        // nothing to sum: norm 0
-  int rc = ensure_partials(ctx, ntiles, st);
-  if (rc != SLIDEDP_OK) return rc;
-  const WholeNorm w{ctx->ticket, ctx->scalars, max_norm, ntiles};
-  const float inv = (float)inv_R;
-  FAULT_POINT();
-  if (R == 1) {
-    grad_norm_whole_r1_kernel<<<(unsigned)((ntiles + kDeepTiles - 1) / kDeepTiles), kNormThreads, 0, st>>>(
-        gp.p[0], n, inv, ctx->partials, w);
-  } else {
-    const unsigned blocks = (unsigned)ntiles;
-    switch (R) {
-#define SLIDEDP_CASE(r)                                                                          \
-  case r:                                                                                        \
-    grad_norm_whole_kernel<r><<<blocks, kNormThreads, 0, st>>>(gp, n, inv, ctx->partials, w);    \
-    break;
-      SLIDEDP_CASE(2) SLIDEDP_CASE(3) SLIDEDP_CASE(4) SLIDEDP_CASE(5) SLIDEDP_CASE(6)
-      SLIDEDP_CASE(7) SLIDEDP_CASE(8) SLIDEDP_CASE(9) SLIDEDP_CASE(10) SLIDEDP_CASE(11)
-      SLIDEDP_CASE(12) SLIDEDP_CASE(13) SLIDEDP_CASE(14) SLIDEDP_CASE(15) SLIDEDP_CASE(16)
-#undef SLIDEDP_CASE
-      default: return SLIDEDP_ERR_INVALID_ARG;
-    }
-  }
-  ctx->launches += 1;
-  CU_AFTER_LAUNCH();
-  ctx->partials_used = ntiles;
-  ctx->norm_issued = true;
-  return SLIDEDP_OK;
-}
-
 // Copies the four scalars to the pinned mirror on `st` and waits (bounded) for them.
 static int fetch_scalars(slidedp_ctx* ctx, cudaStream_t st) {
   CU(cudaMemcpyAsync(ctx->host_scalars, ctx->scalars, 4 * sizeof(double),
@@ -201,27 +166,6 @@ int slidedp_grad_norm_finish(slidedp_ctx* ctx, double max_norm, double* host_nor
   if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   int rc = norm_finish(ctx, max_norm, st);
-  if (rc != SLIDEDP_OK) return rc;
-  if (host_norm || host_coef) {
-    rc = fetch_scalars(ctx, st);
-    if (rc != SLIDEDP_OK) return rc;
-    if (host_norm) *host_norm = ctx->host_scalars[1];
-    if (host_coef) *host_coef = ctx->host_scalars[2];
-  }
-  return SLIDEDP_OK;
-}
-
-int slidedp_grad_norm_whole(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n,
-                            double inv_R, double max_norm, double* host_norm, double* host_coef,
-                            void* cuda_stream) {
-  if (!ctx || n < 0 || inv_R != inv_R || max_norm != max_norm) return SLIDEDP_ERR_INVALID_ARG;
-  GradPtrs gp;
-  int rc = check_grads(grads_bf16, R, &gp);
-  if (rc != SLIDEDP_OK) return rc;
-  DeviceGuard guard(ctx->device);
-  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  rc = norm_whole(ctx, gp, R, n, inv_R, max_norm, st);
   if (rc != SLIDEDP_OK) return rc;
   if (host_norm || host_coef) {
     rc = fetch_scalars(ctx, st);

@@ -81,10 +81,6 @@ _lib.slidedp_grad_norm.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, ctype
 _lib.slidedp_grad_norm_finish.restype = ctypes.c_int
 _lib.slidedp_grad_norm_finish.argtypes = [_vp, ctypes.c_double, ctypes.POINTER(ctypes.c_double),
                                           ctypes.POINTER(ctypes.c_double), _vp]
-_lib.slidedp_grad_norm_whole.restype = ctypes.c_int
-_lib.slidedp_grad_norm_whole.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, ctypes.c_double,
-                                         ctypes.c_double, ctypes.POINTER(ctypes.c_double),
-                                         ctypes.POINTER(ctypes.c_double), _vp]
 _lib.slidedp_grad_norm_tiles.restype = ctypes.c_int
 _lib.slidedp_grad_norm_tiles.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, ctypes.c_double, _vp, _vp]
 _lib.slidedp_grad_norm_finish_from.restype = ctypes.c_int
@@ -250,19 +246,6 @@ class Context:
                                                       ctypes.byref(coef), _stream(stream)))
             return norm.value, coef.value
         self._check(_lib.slidedp_grad_norm_finish(self._h, max_norm, None, None, _stream(stream)))
-        return None
-
-    def slidedp_grad_norm_whole(self, grads, n: int, inv_R: float, max_norm: float,
-                                fetch: bool = False, stream=None):
-        """Norm and coefficient of a single-chunk step in one launch; (norm, coef) if ``fetch``."""
-        if fetch:
-            norm, coef = ctypes.c_double(), ctypes.c_double()
-            self._check(_lib.slidedp_grad_norm_whole(self._h, _grad_array(grads), len(grads), n, inv_R,
-                                                     max_norm, ctypes.byref(norm), ctypes.byref(coef),
-                                                     _stream(stream)))
-            return norm.value, coef.value
-        self._check(_lib.slidedp_grad_norm_whole(self._h, _grad_array(grads), len(grads), n, inv_R,
-                                                 max_norm, None, None, _stream(stream)))
         return None
 
     def slidedp_grad_norm_tiles(self, grads, n: int, inv_R: float, tile_sums_out, stream=None) -> None:

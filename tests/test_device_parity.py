@@ -506,39 +506,3 @@ def test_hbm_mix_probe_leaves_the_state_unchanged(ctx, sd):
     with pytest.raises(sd.SlideDPError) as e:
         ctx.slidedp_hbm_mix_probe(dg, 2, dw, dm, dv, scratch, 3)
     assert e.value.status == sd.ERR_INVALID_ARG
-
-
-@pytest.mark.parametrize("R,n", [(1, 16384 * 37 + 4321), (1, 16384 * 2), (1, 5), (2, 16384 * 21 + 8),
-                                 (4, 16384 * 300 + 77), (8, 16384 * 5 + 9), (13, 16384 + 1), (4, 0)])
-def test_one_launch_norm_has_the_bits_of_the_two_pass_norm(ctx, sd, R, n):
-    """slidedp_grad_norm_whole folds the tile sums in the block that finishes last; which block
-    that is varies, the result must not: same bits as slidedp_grad_norm + slidedp_grad_norm_finish,
-    call after call (the block counter returns to zero by itself), and one kernel launch."""
-    grads, *_ = random_case(max(n, 8), R, seed=3 * R + n % 101, sigma=2e-3)
-    dg = [g.cuda() for g in grads]
-    ctx.slidedp_grad_norm(dg, n, 1.0 / R, True)
-    want = ctx.slidedp_grad_norm_finish(0.3, fetch=True)
-    before = ctx.slidedp_kernel_launches()
-    for _ in range(4):
-        assert ctx.slidedp_grad_norm_whole(dg, n, 1.0 / R, 0.3, fetch=True) == want
-    assert ctx.slidedp_kernel_launches() == before + 4
-    if n:
-        S = oracle.grad_sumsq([parity.u16(g)[:n] for g in grads], 1.0 / R)
-        coef_o, norm_o = oracle.clip_coef(S, 0.3)
-        parity.assert_norm_close(want[0], norm_o)
-        assert abs(want[1] - coef_o) <= 1e-6 * coef_o
-    # and an update that follows uses the coefficient it left in the context
-    if n:
-        _, w, m, v = random_case(n, 1, seed=5)
-        a = [w.cuda(), m.cuda(), v.cuda()]
-        b = [w.cuda(), m.cuda(), v.cuda()]
-        pa, pb = (torch.zeros(n, dtype=torch.bfloat16, device="cuda") for _ in range(2))
-        dgn = [g[:n] for g in dg]
-        hp = sd.HParams(inv_R=1.0 / R, max_norm=0.3, step=2)
-        ctx.slidedp_grad_norm(dgn, n, 1.0 / R, True)
-        ctx.slidedp_grad_norm_finish(0.3)
-        ctx.slidedp_reduce_adamw_chunk(dgn, n, *a, pa, hp)
-        ctx.slidedp_grad_norm_whole(dgn, n, 1.0 / R, 0.3)
-        ctx.slidedp_reduce_adamw_chunk(dgn, n, *b, pb, hp)
-        torch.cuda.synchronize()
-        assert all(torch.equal(x, y) for x, y in zip(a, b)) and torch.equal(pa, pb)

@@ -149,6 +149,27 @@ def run_reference(args):
     return 0
 
 
+class ResultChannel:
+    """The contract is ONE JSON line on stdout. Libraries underneath (NCCL prints its version
+    banner on stdout when a communicator is created) must not add to it: the real stdout is kept
+    aside for the result line and file descriptor 1 points at stderr for everything else."""
+
+    def __init__(self):
+        sys.stdout.flush()
+        self._fd = os.dup(1)
+        os.dup2(2, 1)
+
+    def emit(self, obj) -> None:
+        sys.stdout.flush()
+        with os.fdopen(os.dup(self._fd), "w") as out:
+            out.write(json.dumps(obj) + "\n")
+
+    def close(self) -> None:
+        sys.stdout.flush()
+        os.dup2(self._fd, 1)
+        os.close(self._fd)
+
+
 # ------------------------------------------------------------------ multi-rank plumbing
 def layer_of_rank(rank: int) -> int:
     """Every rank owns a different layer (an independent partition of the model)."""
@@ -186,6 +207,7 @@ def run_cuda(args):
     if not torch.cuda.is_available() or local >= torch.cuda.device_count():
         raise SystemExit("bench.py needs a CUDA device per rank: libslidedp has no CPU path "
                          "(use --impl reference for the CPU oracle)")
+    channel = ResultChannel()
     torch.cuda.set_device(local)
     # under a launcher (torchrun sets RANK and MASTER_ADDR) the process group is used even for
     # one rank, so that the N = 1 run exercises the same barrier / reduction code as N > 1
@@ -345,7 +367,8 @@ def run_cuda(args):
         dist.barrier()
         dist.destroy_process_group()
     if out is not None:
-        print(json.dumps(out))
+        channel.emit(out)
+    channel.close()
     return 0
 
 
@@ -368,6 +391,7 @@ def run_sharded(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available() or local >= torch.cuda.device_count():
         raise SystemExit("bench.py --sharded needs one CUDA device per rank: libslidedp has no CPU path")
+    channel = ResultChannel()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if "MASTER_ADDR" not in os.environ:
@@ -412,7 +436,7 @@ def run_sharded(args):
     if rank == 0:
         # per parameter and rank: (12 + 14)/N state bytes locally, 2 (R - 1)/N gradient bytes
         # and 2 (N - 1)/N parameter bytes over the GPU interconnect, plus the norm's re-read
-        print(json.dumps({
+        channel.emit({
             "metric": METRIC, "value": n * args.steps / (total_ms * 1e-3) / 1e9, "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "strong",
@@ -421,9 +445,10 @@ def run_sharded(args):
                        "parallelism": f"one layer sharded over {world} rank(s): peer-mapped gradient "
                                       "reads, BF16 copy stored to every rank, host barriers"},
             "gpu_launches": launches, "clocks": clocks,
-            "interconnect_bytes_per_rank_per_step": (4 * (R - 1) + 2 * (world - 1)) * (hi - lo)}))
+            "interconnect_bytes_per_rank_per_step": (4 * (R - 1) + 2 * (world - 1)) * (hi - lo)})
     dist.barrier()
     dist.destroy_process_group()
+    channel.close()
     return 0
 
 
@@ -893,9 +918,24 @@ def launch_ranks(world: int, worker, args) -> int:
              for r in range(world)]
     for p in procs:
         p.start()
+    # a rank that dies (no device, a failed check) must not leave the others waiting at the
+    # rendezvous: stop exactly the processes started here as soon as one exits non-zero
+    failed = None
+    while failed is None and any(p.is_alive() for p in procs):
+        for p in procs:
+            p.join(timeout=0.2)
+            if p.exitcode not in (None, 0):
+                failed = p.exitcode
+                break
+    if failed is not None:
+        for p in procs:
+            if p.is_alive():
+                p.terminate()
+        for p in procs:
+            p.join(timeout=10)
+        return failed if failed > 0 else 1
     for p in procs:
         p.join()
-    for p in procs:
         if p.exitcode != 0:
             return p.exitcode if p.exitcode and p.exitcode > 0 else 1
     return 0

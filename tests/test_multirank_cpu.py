@@ -104,3 +104,33 @@ def test_gpus_flag_reaches_the_rank_spawn_and_must_agree_with_a_launcher():
     r = subprocess.run(exe + ["--gpus", "2"], env=dict(env, RANK="0", WORLD_SIZE="4"),
                        capture_output=True, text=True, timeout=120)
     assert r.returncode == 2 and "disagrees with WORLD_SIZE" in r.stderr
+
+
+def _one_rank_dies(args):
+    """Rank 1 fails at once; rank 0 would wait a long time (as it would at a rendezvous)."""
+    if int(os.environ["RANK"]) == 1:
+        return 7
+    import time
+    time.sleep(120)
+    return 0
+
+
+def test_a_failed_rank_does_not_leave_the_others_waiting():
+    import time
+    sys.path.insert(0, ROOT)
+    import bench
+    t0 = time.perf_counter()
+    assert bench.launch_ranks(2, _one_rank_dies, None) == 7
+    assert time.perf_counter() - t0 < 60
+
+
+def test_only_the_result_line_reaches_stdout():
+    """Whatever a library underneath writes to file descriptor 1 (NCCL prints a version banner
+    there) ends up on stderr; stdout carries the one JSON line."""
+    code = ("import os, sys; sys.path.insert(0, %r); import bench\n"
+            "ch = bench.ResultChannel()\n"
+            "os.write(1, b'banner from a C library\\n'); print('a stray print')\n"
+            "ch.emit({'value': 1.5}); ch.close()\n") % ROOT
+    r = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0 and r.stdout == '{"value": 1.5}\n', (r.stdout, r.stderr)
+    assert "banner from a C library" in r.stderr and "a stray print" in r.stderr

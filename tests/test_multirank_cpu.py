@@ -99,8 +99,9 @@ def test_gpus_flag_reaches_the_rank_spawn_and_must_agree_with_a_launcher():
     if not torch.cuda.is_available():
         r = subprocess.run(exe + ["--gpus", "2", "--steps", "1", "--warmup", "0"], env=env,
                            capture_output=True, text=True, timeout=300)
-        # two ranks were started and each stopped where the CUDA path must: no device, no fallback
-        assert r.returncode != 0 and r.stderr.count("needs a CUDA device") == 2, r.stderr
+        # the ranks were started and stopped where the CUDA path must: no device, no fallback
+        # (the first rank to fail takes its sibling down, so one or two messages)
+        assert r.returncode != 0 and 1 <= r.stderr.count("needs a CUDA device") <= 2, r.stderr
     r = subprocess.run(exe + ["--gpus", "2"], env=dict(env, RANK="0", WORLD_SIZE="4"),
                        capture_output=True, text=True, timeout=120)
     assert r.returncode == 2 and "disagrees with WORLD_SIZE" in r.stderr

@@ -849,7 +849,8 @@ def run_kernel_case(args):
       python bench.py --report kernel --kernel update --params 50331648 --R 4 --launches 4
 
     Kernels: update (fused reduce + AdamW + BF16 emit), norm (tile sums + finish), reduce (rank
-    reduction alone), stream (host-resident step through pinned memory)."""
+    reduction alone), stream (host-resident step through pinned memory), deliver (FP32 H2D + BF16
+    cast)."""
     import torch
 
     import paper_2609_34162_b200.slidedp as sd
@@ -864,7 +865,7 @@ def run_kernel_case(args):
     ctx = sd.slidedp_create(0, 0)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.launches + 1)]
     st = torch.cuda.current_stream()
-    if args.kernel == "stream":
+    if args.kernel in ("stream", "deliver"):
         hw, hm, hv = (torch.empty(n, pin_memory=True) for _ in range(3))
         hw.copy_(w); hm.copy_(m); hv.copy_(v)
     ctx.slidedp_grad_norm(grads, n, 1.0 / R, True)
@@ -880,12 +881,14 @@ def run_kernel_case(args):
             ctx.slidedp_grad_norm_finish(args.clip)
         elif args.kernel == "reduce":
             ctx.slidedp_reduce_mean_bf16(grads, n, 1.0 / R, p)
+        elif args.kernel == "deliver":
+            ctx.slidedp_deliver_params(hw, n, p, 16 << 20, 3, want_stats=False)
         else:
             ctx.slidedp_stream_step(grads, n, hw, hm, hv, p, 16 << 20, 3, hp, want_stats=False)
     ev[args.launches].record(st)
     torch.cuda.synchronize()
     ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.launches)]
-    per = {"update": 26 + 2 * R, "norm": 2 * R, "reduce": 2 * R + 2, "stream": 24}[args.kernel]
+    per = {"update": 26 + 2 * R, "norm": 2 * R, "reduce": 2 * R + 2, "stream": 24, "deliver": 4}[args.kernel]
     print(json.dumps({"report": "kernel", "kernel": args.kernel, "params": n, "R": R,
                       "ms_per_launch": ms, "bytes_per_param": per,
                       "best_gbs": per * n / (min(ms) * 1e6)}))
@@ -951,7 +954,8 @@ def main(argv=None):
     ap.add_argument("--sharded", action="store_true",
                     help="one layer sharded over the ranks (peer-mapped gradients, BF16 copy stored "
                          "to every rank) instead of one independent layer per rank")
-    ap.add_argument("--kernel", choices=["update", "norm", "reduce", "stream"], default="update")
+    ap.add_argument("--kernel", choices=["update", "norm", "reduce", "stream", "deliver"],
+                    default="update")
     ap.add_argument("--params", type=int, default=48 << 20)
     ap.add_argument("--R", type=int, default=4)
     ap.add_argument("--launches", type=int, default=4)

@@ -174,3 +174,34 @@ def test_ipc_argument_errors():
         assert e.value.status == sd.ERR_INVALID_ARG
     finally:
         ctx.slidedp_destroy()
+
+
+@pytest.mark.parametrize("R,n,n_outs", [(1, 5, 3), (4, 4 * 128 * 3 + 3, 16), (16, 100_001, 2), (3, 8, 1)])
+def test_broadcast_update_equals_the_plain_update_for_every_output(R, n, n_outs):
+    """Every output of slidedp_reduce_adamw_chunk_bcast, ragged tail included, carries the bits
+    of the plain update; the state does too; guard bands around every output stay intact."""
+    import paper_2609_34162_b200.slidedp as sd
+    ctx = sd.slidedp_create(0, 0)
+    try:
+        g = torch.Generator(device="cuda").manual_seed(100 * R + n_outs)
+        dg = [(torch.randn(n, generator=g, device="cuda") * 1e-3).to(torch.bfloat16) for _ in range(R)]
+        w = torch.randn(n, generator=g, device="cuda") * 0.02
+        m = torch.randn(n, generator=g, device="cuda") * 3e-4
+        v = torch.randn(n, generator=g, device="cuda").square() * 1e-7
+        a, b = [w.clone(), m.clone(), v.clone()], [w.clone(), m.clone(), v.clone()]
+        pa = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+        pad = 8                                             # keeps every output 16-byte aligned
+        banded = [torch.full((n + 2 * pad,), -7.0, dtype=torch.bfloat16, device="cuda")
+                  for _ in range(n_outs)]
+        hp = sd.HParams(inv_R=1.0 / R, max_norm=0.02, step=9)
+        ctx.slidedp_grad_norm(dg, n, 1.0 / R, True)
+        ctx.slidedp_grad_norm_finish(0.02)
+        ctx.slidedp_reduce_adamw_chunk(dg, n, *a, pa, hp)
+        ctx.slidedp_reduce_adamw_chunk_bcast(dg, n, *b, [x[pad:] for x in banded], hp)
+        torch.cuda.synchronize()
+        assert all(torch.equal(x, y) for x, y in zip(a, b))
+        for x in banded:
+            assert torch.equal(x[pad:pad + n], pa)
+            assert torch.all(x[:pad] == -7.0) and torch.all(x[pad + n:] == -7.0)
+    finally:
+        ctx.slidedp_destroy()

@@ -94,6 +94,10 @@ class ShardedStep:
         """Everything this rank queued is complete, then every rank is here."""
         stream.synchronize()
         dist.barrier(group=self.group)
+        if dist.get_backend(self.group) == "nccl":
+            # an NCCL barrier is itself stream work on torch's current stream: wait for it on
+            # the host, so that the ordering holds whatever stream the step's kernels use
+            torch.cuda.current_stream().synchronize()
 
     def step(self, master_shard, m_shard, v_shard, hp: HParams, stream=None):
         """One update. The rank-local gradients must already be complete on every rank's device

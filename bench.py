@@ -318,10 +318,11 @@ def run_cuda(args):
     t_next += 2
     e2e_steps = max(1, min(args.steps, 10))
     barrier()
-    e2e_ms, wall0, last = 0.0, time.perf_counter(), None
+    e2e_ms, wall0, last, per_step = 0.0, time.perf_counter(), None, []
     for i in range(e2e_steps):
         last = ctx.slidedp_stream_step(grads, n, hw, hm, hv, p, ce, 3, hp(t_next + i))
         e2e_ms += last["ms_total"]
+        per_step.append(last["ms_total"])
     wall = time.perf_counter() - wall0
     barrier()
     t_next += e2e_steps
@@ -329,6 +330,7 @@ def run_cuda(args):
     e2e = {"value": job_value(world, n, e2e_steps, e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": 12 * n, "d2h_bytes_per_step": 12 * n + 32,
            "ms_per_step": e2e_ms / e2e_steps, "wall_ms_per_step": wall / e2e_steps * 1e3,
+           "ms_per_step_median": statistics.median(per_step), "ms_per_step_best": min(per_step),
            "steps": e2e_steps, "chunk_mib": 16, "nbuf": 3,
            "note": "FP32 master/m/v in pinned host memory, copied H2D and back D2H every step; "
                    "gradients and the BF16 copy stay on the device where backward/forward use them",

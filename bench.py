@@ -550,6 +550,21 @@ def run_sweep(args):
             row[name] = {"ms": med, "ms_best": best, "bytes_per_param": per,
                          "gbs": per * n / (med * 1e6), "frac_of_measured_peak": per * n / (med * 1e6) / peak}
         by_R.append(row)
+    # the sharded step's update with its BF16 copy stored to G buffers (all local here: the HBM
+    # cost of the stores alone; on real ranks G - 1 of them cross the GPU interconnect)
+    g4 = pool[:4]
+    h4 = sd.HParams(inv_R=0.25, max_norm=1.0, step=11)
+    extra = [torch.zeros(n, dtype=torch.bfloat16, device=dev) for _ in range(7)]
+    bcast = []
+    for G in (1, 2, 4, 8):
+        outs = [p] + extra[:G - 1]
+        med, best = timed(lambda: ctx.slidedp_reduce_adamw_chunk_bcast(g4, n, w, m, v, outs, h4))
+        per = 26 + 2 * 4 + 2 * (G - 1)
+        bcast.append({"outputs": G, "ms": med, "bytes_per_param": per, "gbs": per * n / (med * 1e6),
+                      "frac_of_measured_peak": per * n / (med * 1e6) / peak})
+    out["broadcast_update_R4"] = {"params": n, "rows": bcast,
+                                  "note": "all outputs in local HBM; one GPU cannot show the interconnect"}
+    del extra
     out["by_rank_count"] = {"params": n, "timing": f"median of {reps} launches, CUDA events, inputs >> L2",
                             "rows": by_R}
     del pool, w, m, v, p

@@ -661,9 +661,20 @@ def run_sweep(args):
         ctx.slidedp_stream_wait()
         async_ms.append((time.perf_counter() - t0) * 1e3)
     ams = statistics.mean(async_ms[1:])
+    # and as ONE call: norm over all layers + every layer streamed (slidedp_stream_layers)
+    one_call = []
+    for t in range(wl.steps + 6, wl.steps + 11):
+        torch.cuda.synchronize()
+        one_call.append(ctx.slidedp_stream_layers(
+            [(grads[l], nl, *state[l], ps[l]) for l in range(L)], ce, 3, hp(wl, t)))
+    oms = statistics.mean(r_["ms_total"] for r_ in one_call[1:])
     out["qwen3_14b_8layers_host"] = {
         "async_layers": {"ms_per_step": ams, "g_params_per_s": wl.numel / ams / 1e6,
                          "link_gbs_each_way": 12.0 * wl.numel / (ams * 1e6)},
+        "one_call_stream_layers": {"ms_per_step": oms, "g_params_per_s": wl.numel / oms / 1e6,
+                                   "link_gbs_each_way": 12.0 * wl.numel / (oms * 1e6),
+                                   "ms_norm": statistics.mean(r_["ms_norm"] for r_ in one_call[1:]),
+                                   "timing": "CUDA events inside the call, norm pass included"},
         "params": wl.numel, "R": R, "layers": L, "steps": wl.steps, "chunk_mib": 64, "nbuf": 3,
         "ms_per_step": ms, "g_params_per_s": wl.numel / ms / 1e6,
         "link_gbs_each_way": 12.0 * wl.numel / (ms * 1e6),

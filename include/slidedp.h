@@ -308,6 +308,27 @@ SLIDEDP_API int slidedp_stream_step_async(slidedp_ctx* ctx, const void* const* g
                               const slidedp_hparams* hp);
 SLIDEDP_API int slidedp_stream_wait(slidedp_ctx* ctx);
 
+/* A whole multi-layer step in one call (paper Sec. 3.3: layers are the unit the update is
+ * released in, and completed layers release their updates while other work continues): when
+ * hp->max_norm > 0 the global norm is taken over the gradients of ALL layers, in layer order,
+ * before any update; then every layer is streamed like slidedp_stream_step_async with that
+ * coefficient, the layers sharing the slot ring back to back; the call returns after the last
+ * copy-out (bounded wait). Every layer's arguments are checked before anything is queued.
+ * layers[l]: grads_bf16 = host array of R device pointers to n BF16 values each; host_master /
+ * host_m / host_v = PINNED, n floats, updated in place; param_bf16_out = device, n BF16. The
+ * result is bit-identical to slidedp_grad_norm over the layers + slidedp_grad_norm_finish + one
+ * slidedp_stream_step(norm_ready = 1) per layer. stats (nullable): norm, clip_coef, ms_total,
+ * ms_norm, the two copy lanes over the whole step, chunks (sum); ms_kernel is not measured. */
+typedef struct {
+  const void* const* grads_bf16;
+  int64_t n;
+  float *host_master, *host_m, *host_v;
+  void* param_bf16_out;
+} slidedp_layer;
+SLIDEDP_API int slidedp_stream_layers(slidedp_ctx* ctx, const slidedp_layer* layers, int num_layers, int R,
+                          int64_t chunk_elems, int nbuf, const slidedp_hparams* hp,
+                          slidedp_stats* stats);
+
 /* ---- parameter delivery: BF16 copy of a host-resident FP32 master -------------------------
  *
  * The step BEFORE the update path (paper Sec. 3.3 "Overlap within a layer": on parameter

@@ -11,6 +11,10 @@ using namespace slidedp::host;
 
 namespace {
 
+// Which timing events an enqueue records: the first chunk's copies, the last chunk's copies, one
+// (middle) chunk's kernel.
+constexpr int kMarkFirst = 1, kMarkLast = 2, kMarkKernel = 4;
+
 
 // Grows the slot allocation to `need` bytes if the budget allows (checked before any work).
 int ensure_slots(slidedp_ctx* ctx, size_t need) {
@@ -71,12 +75,12 @@ int abandon_queued(slidedp_ctx* ctx, int status) {
 int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total, float* host_master,
                    float* host_m, float* host_v, void* param_bf16_out, int64_t chunk_elems,
                    int nbuf, int64_t cap, int norm_ready, const slidedp_hparams* hp,
-                   bool synchronous, bool timed, int64_t nchunks);
+                   bool synchronous, int marks, int64_t nchunks);
 
 int enqueue_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n_total,
                         float* host_master, float* host_m, float* host_v, void* param_bf16_out,
                         int64_t chunk_elems, int nbuf, int norm_ready, const slidedp_hparams* hp,
-                        bool synchronous, bool timed, int64_t* nchunks_out) {
+                        bool synchronous, int marks, int64_t* nchunks_out) {
   if (!ctx || n_total < 0) return SLIDEDP_ERR_INVALID_ARG;
   int rc = check_hparams(hp);
   if (rc != SLIDEDP_OK) return rc;
@@ -122,7 +126,7 @@ int enqueue_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
   }
   const int64_t nchunks = n_total == 0 ? 0 : (n_total + chunk_elems - 1) / chunk_elems;
   *nchunks_out = nchunks;
-  if (timed) {
+  if (marks & kMarkKernel) {
     while (ctx->timing.empty() && nchunks > 0) {
       ChunkEvents c;
       CU(cudaEventCreate(&c.k_start));
@@ -133,7 +137,7 @@ int enqueue_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
 
   ctx->ring_busy = true;
   rc = enqueue_chunks(ctx, gp, R, n_total, host_master, host_m, host_v, param_bf16_out,
-                      chunk_elems, nbuf, cap, norm_ready, hp, synchronous, timed, nchunks);
+                      chunk_elems, nbuf, cap, norm_ready, hp, synchronous, marks, nchunks);
   if (rc != SLIDEDP_OK) return abandon_queued(ctx, rc);
   return SLIDEDP_OK;
 }
@@ -143,7 +147,7 @@ int enqueue_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
 int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total, float* host_master,
                    float* host_m, float* host_v, void* param_bf16_out, int64_t chunk_elems,
                    int nbuf, int64_t cap, int norm_ready, const slidedp_hparams* hp,
-                   bool synchronous, bool timed, int64_t nchunks) {
+                   bool synchronous, int marks, int64_t nchunks) {
   const bool clip = hp->max_norm > 0.0;
   int rc = SLIDEDP_OK;
   if (synchronous) {
@@ -170,15 +174,15 @@ int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total,
     float* sw = ctx->slots + (size_t)slot * 3 * cap;
     float* sm = sw + cap;
     float* sv = sm + cap;
-    ChunkEvents* te = (timed && c == (nchunks - 1) / 2) ? &ctx->timing[0] : nullptr;
+    ChunkEvents* te = ((marks & kMarkKernel) && c == (nchunks - 1) / 2) ? &ctx->timing[0] : nullptr;
     // copy-in: the slot must have been drained by the copy-out that last used it (a no-op
     // for an event that was never recorded or has completed)
     CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_free[slot], 0));
-    if (timed && c == 0) CU(cudaEventRecord(ctx->ev_in_first, ctx->s_in));
+    if ((marks & kMarkFirst) && c == 0) CU(cudaEventRecord(ctx->ev_in_first, ctx->s_in));
     CU(cudaMemcpyAsync(sw, host_master + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
     CU(cudaMemcpyAsync(sm, host_m + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
     CU(cudaMemcpyAsync(sv, host_v + off, bytes, cudaMemcpyHostToDevice, ctx->s_in));
-    if (timed && c == nchunks - 1) CU(cudaEventRecord(ctx->ev_in_last, ctx->s_in));
+    if ((marks & kMarkLast) && c == nchunks - 1) CU(cudaEventRecord(ctx->ev_in_last, ctx->s_in));
     CU(cudaEventRecord(ctx->ev_loaded[slot], ctx->s_in));
     // update
     CU(cudaStreamWaitEvent(ctx->s_compute, ctx->ev_loaded[slot], 0));
@@ -191,11 +195,11 @@ int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total,
     CU(cudaEventRecord(ctx->ev_updated[slot], ctx->s_compute));
     // copy-out
     CU(cudaStreamWaitEvent(ctx->s_out, ctx->ev_updated[slot], 0));
-    if (timed && c == 0) CU(cudaEventRecord(ctx->ev_out_first, ctx->s_out));
+    if ((marks & kMarkFirst) && c == 0) CU(cudaEventRecord(ctx->ev_out_first, ctx->s_out));
     CU(cudaMemcpyAsync(host_master + off, sw, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
     CU(cudaMemcpyAsync(host_m + off, sm, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
     CU(cudaMemcpyAsync(host_v + off, sv, bytes, cudaMemcpyDeviceToHost, ctx->s_out));
-    if (timed && c == nchunks - 1) CU(cudaEventRecord(ctx->ev_out_last, ctx->s_out));
+    if ((marks & kMarkLast) && c == nchunks - 1) CU(cudaEventRecord(ctx->ev_out_last, ctx->s_out));
     CU(cudaEventRecord(ctx->ev_free[slot], ctx->s_out));
   }
   ctx->ring_next += nchunks;
@@ -225,7 +229,7 @@ int slidedp_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
   int64_t nchunks = 0;
   int rc = enqueue_stream_step(ctx, grads_bf16, R, n_total, host_master, host_m, host_v,
                                param_bf16_out, chunk_elems, nbuf, norm_ready, hp,
-                               /*synchronous=*/true, stats != nullptr, &nchunks);
+                               /*synchronous=*/true, stats ? (kMarkFirst | kMarkLast | kMarkKernel) : 0, &nchunks);
   if (rc != SLIDEDP_OK) return rc;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
@@ -273,7 +277,121 @@ int slidedp_stream_step_async(slidedp_ctx* ctx, const void* const* grads_bf16, i
   int64_t nchunks = 0;
   return enqueue_stream_step(ctx, grads_bf16, R, n_total, host_master, host_m, host_v,
                              param_bf16_out, chunk_elems, nbuf, norm_ready, hp,
-                             /*synchronous=*/false, /*timed=*/false, &nchunks);
+                             /*synchronous=*/false, /*marks=*/0, &nchunks);
+}
+
+int slidedp_stream_layers(slidedp_ctx* ctx, const slidedp_layer* layers, int num_layers, int R,
+                          int64_t chunk_elems, int nbuf, const slidedp_hparams* hp,
+                          slidedp_stats* stats) {
+  if (stats) {
+    memset(stats, 0, sizeof *stats);
+    stats->clip_coef = 1.0;
+  }
+  if (!ctx || num_layers < 0 || (num_layers > 0 && !layers)) return SLIDEDP_ERR_INVALID_ARG;
+  int rc = check_hparams(hp);
+  if (rc != SLIDEDP_OK) return rc;
+  const bool clip = hp->max_norm > 0.0;
+  // every layer's arguments are checked before anything is queued
+  int first = -1, last = -1;
+  for (int l = 0; l < num_layers; ++l) {
+    const slidedp_layer& L = layers[l];
+    GradPtrs gp;
+    if (L.n < 0) return SLIDEDP_ERR_INVALID_ARG;
+    rc = check_grads(L.grads_bf16, R, &gp);
+    if (rc != SLIDEDP_OK) return rc;
+    if (L.n > 0 && (!L.host_master || !L.host_m || !L.host_v || !L.param_bf16_out))
+      return SLIDEDP_ERR_INVALID_ARG;
+    if (!aligned16(L.host_master) || !aligned16(L.host_m) || !aligned16(L.host_v) ||
+        !aligned16(L.param_bf16_out))
+      return SLIDEDP_ERR_MISALIGNED;
+    if (L.n > 0) { if (first < 0) first = l; last = l; }
+  }
+  if (nbuf < 2 || nbuf > 3 || chunk_elems <= 0 || (chunk_elems % 8) != 0)
+    return SLIDEDP_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
+  for (int l = 0; l < num_layers; ++l) {
+    if (layers[l].n == 0) continue;
+    for (const float* h : {layers[l].host_master, layers[l].host_m, layers[l].host_v}) {
+      bool pinned = false;
+      rc = is_pinned(ctx, h, &pinned);
+      if (rc != SLIDEDP_OK) return rc;
+      if (!pinned) return SLIDEDP_ERR_NOT_PINNED;
+    }
+  }
+  {
+    int64_t biggest = 0;
+    for (int l = 0; l < num_layers; ++l) if (layers[l].n > biggest) biggest = layers[l].n;
+    const int64_t cap = chunk_elems < biggest ? chunk_elems : ((biggest + 7) / 8) * 8;
+    if (ctx->budget && (size_t)nbuf * 3 * (size_t)cap * sizeof(float) > ctx->budget)
+      return SLIDEDP_ERR_BUDGET;
+  }
+
+  int64_t chunks = 0;
+  ctx->ring_busy = true;
+  auto enqueue = [&]() -> int {
+    CU(cudaEventRecord(ctx->ev_begin, ctx->s_compute));
+    CU(cudaStreamWaitEvent(ctx->s_in, ctx->ev_begin, 0));
+    CU(cudaStreamWaitEvent(ctx->s_out, ctx->ev_begin, 0));
+    if (clip) {
+      // the norm covers every layer of the step before any update (tile sums in layer order)
+      for (int l = 0; l < num_layers; ++l) {
+        GradPtrs gp;
+        check_grads(layers[l].grads_bf16, R, &gp);
+        int r2 = norm_chunk(ctx, gp, R, layers[l].n, hp->inv_R, l == 0, ctx->s_compute);
+        if (r2 != SLIDEDP_OK) return r2;
+      }
+      if (num_layers == 0) ctx->partials_used = 0;
+      int r2 = norm_finish(ctx, hp->max_norm, ctx->s_compute);
+      if (r2 != SLIDEDP_OK) return r2;
+    }
+    CU(cudaEventRecord(ctx->ev_norm_done, ctx->s_compute));
+    for (int l = 0; l < num_layers; ++l) {
+      const slidedp_layer& L = layers[l];
+      int64_t nchunks = 0;
+      const int marks = stats ? ((l == first ? kMarkFirst : 0) | (l == last ? kMarkLast : 0)) : 0;
+      int r2 = enqueue_stream_step(ctx, L.grads_bf16, R, L.n, L.host_master, L.host_m, L.host_v,
+                                   L.param_bf16_out, chunk_elems, nbuf, /*norm_ready=*/1, hp,
+                                   /*synchronous=*/false, marks, &nchunks);
+      if (r2 != SLIDEDP_OK) return r2;
+      chunks += nchunks;
+    }
+    CU(cudaStreamWaitEvent(ctx->s_out, ctx->ev_norm_done, 0));
+    if (clip) CU(cudaMemcpyAsync(ctx->host_scalars, ctx->scalars, 4 * sizeof(double),
+                                 cudaMemcpyDeviceToHost, ctx->s_out));
+    CU(cudaEventRecord(ctx->ev_end, ctx->s_out));
+    return SLIDEDP_OK;
+  };
+  rc = enqueue();
+  if (rc != SLIDEDP_OK) return abandon_queued(ctx, rc);
+  rc = bounded_event_wait(ctx, ctx->ev_end, ctx->wait_seconds);
+  if (rc != SLIDEDP_OK) return rc;
+  rc = drain_streams(ctx);
+  if (rc != SLIDEDP_OK) return rc;
+  if (stats) {
+    float ms = 0.f;
+    int64_t total = 0;
+    for (int l = 0; l < num_layers; ++l) total += layers[l].n;
+    CU(cudaEventElapsedTime(&ms, ctx->ev_begin, ctx->ev_end));
+    stats->ms_total = ms;
+    CU(cudaEventElapsedTime(&ms, ctx->ev_begin, ctx->ev_norm_done));
+    stats->ms_norm = clip ? ms : 0.0;
+    stats->chunks = chunks;
+    if (first >= 0) {
+      CU(cudaEventElapsedTime(&ms, ctx->ev_in_first, ctx->ev_in_last));
+      stats->ms_h2d = ms;
+      CU(cudaEventElapsedTime(&ms, ctx->ev_out_first, ctx->ev_out_last));
+      stats->ms_d2h = ms;
+      if (stats->ms_h2d > 0) stats->gbs_h2d = 12.0 * (double)total / (stats->ms_h2d * 1e6);
+      if (stats->ms_d2h > 0) stats->gbs_d2h = 12.0 * (double)total / (stats->ms_d2h * 1e6);
+    }
+    if (clip) {
+      stats->norm = ctx->host_scalars[1];
+      stats->clip_coef = ctx->host_scalars[2];
+      stats->nonfinite = ctx->host_scalars[3] != 0.0;
+    }
+  }
+  return SLIDEDP_OK;
 }
 
 int slidedp_stream_wait(slidedp_ctx* ctx) {

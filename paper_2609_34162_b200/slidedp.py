@@ -100,6 +100,15 @@ _lib.slidedp_stream_step_async.restype = ctypes.c_int
 _lib.slidedp_stream_step_async.argtypes = [_vp, _pp, ctypes.c_int, ctypes.c_int64, _vp, _vp, _vp, _vp,
                                            ctypes.c_int64, ctypes.c_int, ctypes.c_int,
                                            ctypes.POINTER(_HParams)]
+class _Layer(ctypes.Structure):
+    _fields_ = [("grads_bf16", _pp), ("n", ctypes.c_int64), ("host_master", _vp), ("host_m", _vp),
+                ("host_v", _vp), ("param_bf16_out", _vp)]
+
+
+_lib.slidedp_stream_layers.restype = ctypes.c_int
+_lib.slidedp_stream_layers.argtypes = [_vp, ctypes.POINTER(_Layer), ctypes.c_int, ctypes.c_int,
+                                       ctypes.c_int64, ctypes.c_int, ctypes.POINTER(_HParams),
+                                       ctypes.POINTER(_Stats)]
 _lib.slidedp_stream_wait.restype = ctypes.c_int
 _lib.slidedp_stream_wait.argtypes = [_vp]
 _lib.slidedp_deliver_params.restype = ctypes.c_int
@@ -324,6 +333,24 @@ class Context:
             self._h, _grad_array(grads), len(grads), n_total, _ptr(host_master), _ptr(host_m),
             _ptr(host_v), _ptr(param_bf16_out), chunk_elems, nbuf, int(norm_ready),
             ctypes.byref(c)))
+
+    def slidedp_stream_layers(self, layers, chunk_elems: int, nbuf: int, hp: HParams,
+                              want_stats: bool = True):
+        """``layers``: sequence of (grads, n, host_master, host_m, host_v, param_bf16_out), every
+        ``grads`` a list of the same R device buffers' worth of rank gradients."""
+        R = len(layers[0][0]) if layers else 1
+        keep = [_grad_array(L[0]) for L in layers]              # the pointer arrays must outlive the call
+        arr = (_Layer * max(len(layers), 1))()
+        for i, (L, g) in enumerate(zip(layers, keep)):
+            if len(L[0]) != R:
+                raise ValueError("every layer needs the same number of rank gradients")
+            arr[i] = _Layer(ctypes.cast(g, _pp), L[1], _ptr(L[2]), _ptr(L[3]), _ptr(L[4]), _ptr(L[5]))
+        c, st = hp._c(), _Stats()
+        self._check(_lib.slidedp_stream_layers(self._h, arr, len(layers), R, chunk_elems, nbuf,
+                                               ctypes.byref(c), ctypes.byref(st) if want_stats else None))
+        if not want_stats:
+            return None
+        return {f: getattr(st, f) for f, _ in _Stats._fields_ if f != "reserved"}
 
     def slidedp_stream_wait(self) -> None:
         self._check(_lib.slidedp_stream_wait(self._h))

@@ -176,6 +176,20 @@ def test_every_streaming_entry_point_survives_a_failed_runtime_call(ctx, sd):
     assert _sweep(ctx, sd, async_step, usable) >= 3 * 12
     case.check_state(*(h.numpy() for h in state["h"]), parity.u16(state["p"]))
 
+    # the multi-layer step: two layers (the two halves of the case), one global norm
+    half = (n // 2) // 8 * 8
+
+    def layers_step():
+        fresh()
+        h, p = state["h"], state["p"]
+        ctx.slidedp_stream_layers(
+            [([g[:half] for g in case.dg], half, h[0][:half], h[1][:half], h[2][:half], p[:half]),
+             ([g[half:] for g in case.dg], n - half, h[0][half:], h[1][half:], h[2][half:], p[half:])],
+            4096, 3, hp)
+
+    assert _sweep(ctx, sd, layers_step, usable) >= 6 * 14
+    case.check_state(*(h.numpy() for h in state["h"]), parity.u16(state["p"]))
+
     # parameter delivery
     master = pinned(case.ow)
     out = torch.zeros(n, dtype=torch.bfloat16, device="cuda")

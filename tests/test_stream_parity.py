@@ -319,6 +319,62 @@ def test_async_layers_share_the_slot_ring_and_match_the_synchronous_step(ctx, sd
     ctx.slidedp_stream_wait()
 
 
+def test_multi_layer_step_in_one_call_matches_the_per_layer_calls(ctx, sd):
+    """slidedp_stream_layers (global norm over every layer, then all layers streamed back to back)
+    against slidedp_grad_norm per layer + finish + one synchronous slidedp_stream_step per layer:
+    same norm, coefficient, state and BF16 copies, bit for bit; layers of different sizes,
+    including an empty one and one smaller than a chunk."""
+    wl = W.scaled(W.CONFIGS["qwen3_14b_8layers_host"], 64)
+    R, nl = wl.R, wl.layer_numel
+    sizes = [nl, nl - 12345, 0, 70_001, nl]
+    L = len(sizes)
+    kw = dict(inv_R=1.0 / R, max_norm=wl.max_norm, step=2, **wl.hparams)
+    dg = [[W.rank_gradient(wl, r, step=2, layer=l, device="cuda")[:max(sizes[l], 8)].clone()
+           for r in range(R)] for l in range(L)]
+    init = [[parity.f32(W.master_weights(wl, layer=l, device="cuda"))[:sizes[l]].copy(),
+             np.full(sizes[l], 1e-4, np.float32), np.full(sizes[l], 1e-7, np.float32)] for l in range(L)]
+    ce = 1 << 19
+
+    def state():
+        host = [[pinned(a) if a.size else torch.empty(8, pin_memory=True)[:0] for a in init[l]]
+                for l in range(L)]
+        dp = [torch.zeros(max(sizes[l], 8), dtype=torch.bfloat16, device="cuda") for l in range(L)]
+        torch.cuda.synchronize()
+        return host, dp
+
+    host_a, dp_a = state()
+    for l in range(L):
+        ctx.slidedp_grad_norm(dg[l], sizes[l], kw["inv_R"], l == 0)
+    norm, coef = ctx.slidedp_grad_norm_finish(wl.max_norm, fetch=True)
+    for l in range(L):
+        ctx.slidedp_stream_step(dg[l], sizes[l], *host_a[l], dp_a[l], ce, 3, sd.HParams(**kw),
+                                norm_ready=True, want_stats=False)
+    host_b, dp_b = state()
+    st = ctx.slidedp_stream_layers([(dg[l], sizes[l], *host_b[l], dp_b[l]) for l in range(L)], ce, 3,
+                                   sd.HParams(**kw))
+    assert (st["norm"], st["clip_coef"]) == (norm, coef) and coef < 1.0
+    assert st["chunks"] == sum(-(-n // ce) for n in sizes) and st["ms_total"] > 0
+    for l in range(L):
+        for a, b in zip(host_a[l], host_b[l]):
+            assert np.array_equal(a.numpy(), b.numpy())
+        assert torch.equal(dp_a[l], dp_b[l])
+    # without clipping, and with no layers at all
+    host_c, dp_c = state()
+    ctx.slidedp_stream_layers([(dg[l], sizes[l], *host_c[l], dp_c[l]) for l in range(L)], ce, 2,
+                              sd.HParams(**dict(kw, max_norm=0.0)), want_stats=False)
+    assert not np.array_equal(host_c[0][0].numpy(), host_b[0][0].numpy())
+    st0 = ctx.slidedp_stream_layers([], ce, 3, sd.HParams(**kw))
+    assert st0["chunks"] == 0 and st0["norm"] == 0.0 and st0["clip_coef"] == 1.0
+    # one bad layer stops the call before any layer is touched
+    host_d, dp_d = state()
+    bad = [(dg[l], sizes[l], *host_d[l], dp_d[l]) for l in range(L)]
+    bad[3] = (dg[3], sizes[3], torch.zeros(sizes[3]), host_d[3][1], host_d[3][2], dp_d[3])   # pageable
+    with pytest.raises(sd.SlideDPError) as e:
+        ctx.slidedp_stream_layers(bad, ce, 3, sd.HParams(**kw))
+    assert e.value.status == sd.ERR_NOT_PINNED
+    assert np.array_equal(host_d[0][0].numpy(), init[0][0])
+
+
 def test_zero_copy_update_on_pinned_host_state_matches_the_device_path(ctx, sd):
     """With unified addressing the fused kernel can read and write pinned host state directly
     (no slots at all): same bits as the device-resident update."""

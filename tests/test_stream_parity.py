@@ -167,15 +167,16 @@ def eight_layers_ten_steps(ctx, sd, wl, ce, restart_steps):
     torch.cuda.synchronize()
     for t in range(1, wl.steps + 1):
         kw = dict(inv_R=1.0 / R, max_norm=wl.max_norm, step=t, **wl.hparams)
-        # ---- CUDA path: norm over all layers, then every layer streamed
+        # ---- CUDA path: the whole step as one call (norm over all layers, then every layer
+        # streamed back to back); the single-layer restarts below use slidedp_stream_step
         for l in range(L):
             for r in range(R):
                 W.rank_gradient(wl, r, step=t, layer=l, device="cuda", out=dg[l][r])
-            ctx.slidedp_grad_norm(dg[l], nl, kw["inv_R"], l == 0)
-        norm_g, coef_g = ctx.slidedp_grad_norm_finish(wl.max_norm, fetch=True)
-        for l in range(L):
-            ctx.slidedp_stream_step(dg[l], nl, host[l][0], host[l][1], host[l][2], dp[l], ce, 3,
-                                    sd.HParams(**kw), norm_ready=True, want_stats=False)
+        torch.cuda.synchronize()
+        st = ctx.slidedp_stream_layers([(dg[l], nl, host[l][0], host[l][1], host[l][2], dp[l])
+                                        for l in range(L)], ce, 3, sd.HParams(**kw))
+        norm_g, coef_g = st["norm"], st["clip_coef"]
+        assert st["chunks"] == L * -(-nl // ce)
         # ---- oracle: sum of squares over all layers first, then the update, layer by layer
         order = list(range(L)) * 2                       # pass A (norm), pass B (update)
         stage.prefetch(0, dg[order[0]])

@@ -91,6 +91,32 @@ int main(void) {
   CHECK_SD(slidedp_stream_step_async(ctx, (const void* const*)dg, R, n, qw, qm, qv, dp4, 4096, 2, 1, &hp_sd));
   CHECK_SD(slidedp_stream_wait(ctx));
   const int async_same = memcmp(qw, pw, n * 4) == 0 && memcmp(qm, pm, n * 4) == 0 && memcmp(qv, pv, n * 4) == 0;
+  /* the step once more as a two-layer call (the two halves of the chunk, one global norm) */
+  float *rw, *rm, *rv;
+  void* dp5;
+  CHECK_CUDA(cudaMallocHost((void**)&rw, n * 4)); CHECK_CUDA(cudaMallocHost((void**)&rm, n * 4));
+  CHECK_CUDA(cudaMallocHost((void**)&rv, n * 4)); CHECK_CUDA(cudaMalloc(&dp5, n * 2));
+  memcpy(rw, hw, n * 4); memcpy(rm, hm, n * 4); memcpy(rv, hv, n * 4);
+  const int64_t half = 50000;                       /* a multiple of 8: both halves stay aligned */
+  const void* g0[R]; const void* g1[R];
+  for (int r = 0; r < R; ++r) { g0[r] = dg[r]; g1[r] = (const uint16_t*)dg[r] + half; }
+  slidedp_layer layers[2] = {{g0, half, rw, rm, rv, dp5},
+                             {g1, n - half, rw + half, rm + half, rv + half, (uint16_t*)dp5 + half}};
+  slidedp_stats lst;
+  CHECK_SD(slidedp_stream_layers(ctx, layers, 2, R, 8192, 3, &hp_sd, &lst));
+  /* the layer cut is not at a norm-tile boundary, so the norm agrees to rounding (not to the
+   * bit) and the state is compared under the benchmark's tolerance */
+  int64_t layers_bad = 0;
+  const float *la[3] = {rw, rm, rv}, *lb[3] = {pw, pm, pv};
+  for (int a = 0; a < 3; ++a)
+    for (int64_t i = 0; i < n; ++i)
+      if (!(fabs((double)la[a][i] - lb[a][i]) <= fmax(1e-6 * fabs((double)lb[a][i]), 1e-12))) ++layers_bad;
+  const int layers_same = layers_bad == 0 && fabs(lst.norm - norm) <= 1e-12 * norm &&
+                          lst.chunks == (half + 8191) / 8192 + (n - half + 8191) / 8192;
+  slidedp_ipc_handle ih;
+  CHECK_SD(slidedp_ipc_export(ctx, (const char*)dp5 + 64, &ih));
+  double mix_gbs = 0;
+  CHECK_SD(slidedp_hbm_mix_probe(ctx, (const void* const*)dg, R, n, dw, dm, dv, dp5, 2, &mix_gbs, NULL));
   double link[4] = {0, 0, 0, 0};
   CHECK_SD(slidedp_link_probe(ctx, qm, qv, dw, dm, (size_t)n * 4, 65536, 1, link));
   uint16_t *gp2 = malloc(n * 2), *gp3 = malloc(n * 2), *want3 = malloc(n * 2);
@@ -122,7 +148,7 @@ int main(void) {
   host_differs += memcmp(gp2, gp, n * 2) != 0;
   oracle_cast_master_to_bf16(pw, n, want3);
   for (int64_t i = 0; i < n; ++i) delivery_differs += gp3[i] != want3[i];
-  const int host_ok = async_same && link[0] > 0 && link[1] > 0 && link[2] > 0 && link[3] > 0 &&
+  const int host_ok = layers_same && ih.offset >= 64 && mix_gbs > 0 && async_same && link[0] > 0 && link[1] > 0 && link[2] > 0 && link[3] > 0 &&
                       host_differs == 0 && delivery_differs == 0 && st.chunks == (n + 8191) / 8192 &&
                       st.norm == norm && st.clip_coef == coef && dst.chunks == (n + 16383) / 16384;
   const int ok = bad == 0 && bf16_differ <= n / 10000 && fabs(norm - onorm) <= 1e-6 * onorm &&

@@ -401,35 +401,44 @@ scatter_tile_sums_kernel(const double* __restrict__ src, int64_t count, F64Dsts 
 // (float)1/R as the fused kernel, then one round-to-nearest-even to BF16. Eight elements per
 // thread; 2R + 2 bytes of traffic per parameter.
 constexpr int kReduceThreads = 256;
-template <int R>
+// U = 16-byte loads per rank in flight per thread: 1 for R >= 2; 2 at R = 1, where a thread's 8
+// elements are only 16 bytes and the kernel was latency-bound (5.7 -> 6.4 TB/s at 100 M
+// parameters; the 32-byte load form of the same shape measured the same, so plain 16-byte
+// accesses are kept).
+template <int R, int U = (R == 1) ? 2 : 1>
 __global__ void __launch_bounds__(kReduceThreads)
 reduce_mean_bf16_kernel(GradPtrs gp, int64_t n, float inv_R, uint16_t* __restrict__ out) {
-  const int64_t base = ((int64_t)blockIdx.x * kReduceThreads + threadIdx.x) * 8;
+  const int64_t base = ((int64_t)blockIdx.x * kReduceThreads + threadIdx.x) * (8 * U);
   if (base >= n) return;
-  if (base + 8 <= n) {
-    uint4 graw[R];
+  if (base + 8 * U <= n) {
+    uint4 graw[U][R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) graw[r] = ld_stream(gp.p[r] + base);
-    float s[8];
-    {
-      const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[0]);
+    for (int u = 0; u < U; ++u)
 #pragma unroll
-      for (int j = 0; j < 4; ++j) { s[2 * j] = bf16_lo(x[j]); s[2 * j + 1] = bf16_hi(x[j]); }
-    }
+      for (int r = 0; r < R; ++r) graw[u][r] = ld_stream(gp.p[r] + base + 8 * u);
 #pragma unroll
-    for (int r = 1; r < R; ++r) {
-      const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[r]);
+    for (int u = 0; u < U; ++u) {
+      float s[8];
+      {
+        const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[u][0]);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        s[2 * j] = __fadd_rn(s[2 * j], bf16_lo(x[j]));
-        s[2 * j + 1] = __fadd_rn(s[2 * j + 1], bf16_hi(x[j]));
+        for (int j = 0; j < 4; ++j) { s[2 * j] = bf16_lo(x[j]); s[2 * j + 1] = bf16_hi(x[j]); }
       }
-    }
-    uint32_t b[8];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) b[j] = f32_to_bf16_bits(__fmul_rn(s[j], inv_R));
-    st_stream(out + base, make_uint4(b[0] | (b[1] << 16), b[2] | (b[3] << 16),
-                                     b[4] | (b[5] << 16), b[6] | (b[7] << 16)));
+      for (int r = 1; r < R; ++r) {
+        const uint32_t* x = reinterpret_cast<const uint32_t*>(&graw[u][r]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          s[2 * j] = __fadd_rn(s[2 * j], bf16_lo(x[j]));
+          s[2 * j + 1] = __fadd_rn(s[2 * j + 1], bf16_hi(x[j]));
+        }
+      }
+      uint32_t b[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) b[j] = f32_to_bf16_bits(__fmul_rn(s[j], inv_R));
+      st_stream(out + base + 8 * u, make_uint4(b[0] | (b[1] << 16), b[2] | (b[3] << 16),
+                                               b[4] | (b[5] << 16), b[6] | (b[7] << 16)));
+    }
   } else {
     for (int64_t i = base; i < n; ++i) {
       float t = __uint_as_float((uint32_t)gp.p[0][i] << 16);

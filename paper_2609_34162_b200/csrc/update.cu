@@ -356,7 +356,8 @@ int slidedp_reduce_mean_bf16(slidedp_ctx* ctx, const void* const* grads_bf16, in
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const unsigned blocks = (unsigned)((n + 8 * kReduceThreads - 1) / (8 * kReduceThreads));
+  const int64_t per_block = (R == 1 ? 16 : 8) * (int64_t)kReduceThreads;   // elements per block
+  const unsigned blocks = (unsigned)((n + per_block - 1) / per_block);
   uint16_t* out = static_cast<uint16_t*>(out_bf16);
   const float inv = (float)inv_R;
   FAULT_POINT();

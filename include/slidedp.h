@@ -110,8 +110,8 @@ SLIDEDP_API int slidedp_destroy(slidedp_ctx* ctx);
  * (after raising the bound or simply later) returns SLIDEDP_OK once they are done, after which
  * the context is as usable as before and the step's results are complete.
  *
- * SLIDEDP_ERR_CUDA from a streaming entry point (slidedp_stream_step, _async, slidedp_deliver_params,
- * slidedp_link_probe) means a runtime call failed midway through enqueuing. Before returning, the
+ * SLIDEDP_ERR_CUDA from a streaming entry point (slidedp_stream_step, _async, slidedp_stream_layers,
+ * slidedp_deliver_params, slidedp_link_probe) means a runtime call failed midway through enqueuing. Before returning, the
  * entry point waits (bounded) for the part it had already queued, so no copy touches the
  * caller's memory after the return, and restarts its slot ring; the context stays usable. The
  * host state is then partly updated: chunks queued before the failure carry the new values, the

@@ -27,4 +27,13 @@ __device__ __forceinline__ void st_stream(void* p, uint4 v) {
   __stcs(reinterpret_cast<uint4*>(p), v);
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization
+// attribute may be scheduled while the kernel before it in the stream is still finishing; this
+// wait holds it until that kernel has completed and its writes are visible. Launched the plain
+// way the instruction does nothing. Every kernel that can be launched that way executes it
+// before its first global-memory access.
+__device__ __forceinline__ void wait_for_previous_kernel() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 }  // namespace slidedp

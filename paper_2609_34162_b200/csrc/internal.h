@@ -123,7 +123,7 @@ UpdateConsts make_consts(const slidedp_hparams* hp);
 // Kernel launchers (update.cu), used by the device-resident entry points and the slot ring.
 int launch_update(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, float* w, float* m,
                   float* v, uint16_t* p, const UpdateConsts& k, const double* coef,
-                  cudaStream_t st);
+                  cudaStream_t st, bool early);
 void launch_sumsq(const GradPtrs& gp, int R, int64_t n, float inv_R, double* tile_sums,
                   unsigned blocks, cudaStream_t st);
 int norm_chunk(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, double inv_R,

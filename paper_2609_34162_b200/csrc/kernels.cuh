@@ -110,6 +110,7 @@ __device__ __forceinline__ void reduce_adamw_body(const GradPtrs& gp, int64_t n,
                                                   const double* __restrict__ clip_coef) {
   const int64_t base = ((int64_t)blockIdx.x * kUpdateThreads + threadIdx.x) * kVec;
   if (base >= n) return;
+  wait_for_previous_kernel();      // the clip coefficient and the state come from earlier kernels
   const double c = clip_coef ? *clip_coef : 1.0;
   const double k1 = k.omb1 * c, k2 = k.omb2 * c * c;
 
@@ -356,6 +357,7 @@ __global__ void __launch_bounds__(kFinishThreads)
 grad_norm_finish_kernel(const double* __restrict__ partials, int64_t count, double max_norm,
                         double* __restrict__ scalars) {
   __shared__ double warp_sum[kFinishThreads / 32];
+  wait_for_previous_kernel();      // the tile sums come from the kernel(s) before this one
   double acc = 0.0;
   for (int64_t i = threadIdx.x; i < count; i += kFinishThreads) acc += partials[i];
 #pragma unroll

@@ -189,7 +189,8 @@ int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total,
     if (te) CU(cudaEventRecord(te->k_start, ctx->s_compute));
     GradPtrs gc = gp;
     for (int r = 0; r < R; ++r) gc.p[r] = gp.p[r] + off;
-    rc = launch_update(ctx, gc, R, len, sw, sm, sv, pout + off, k, coef, ctx->s_compute);
+    rc = launch_update(ctx, gc, R, len, sw, sm, sv, pout + off, k, coef, ctx->s_compute,
+                       /*early=*/false);
     if (rc != SLIDEDP_OK) return rc;
     if (te) CU(cudaEventRecord(te->k_end, ctx->s_compute));
     CU(cudaEventRecord(ctx->ev_updated[slot], ctx->s_compute));

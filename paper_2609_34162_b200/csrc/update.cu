@@ -12,23 +12,43 @@ using namespace slidedp::host;
 namespace slidedp {
 namespace host {
 
+// Launch configuration for a kernel that may start being scheduled while the previous kernel
+// of the stream is finishing (programmatic dependent launch; the kernel itself waits for that
+// kernel's completion before touching memory). `early` = false is a plain launch.
+struct LaunchCfg {
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  LaunchCfg(unsigned blocks, unsigned threads, cudaStream_t st, bool early) {
+    cfg = cudaLaunchConfig_t{};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(threads);
+    cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = early ? 1 : 0;
+  }
+};
+
 template <int R_T>
 static void launch_update_t(const GradPtrs& gp, int /*R*/, int64_t n, float* w, float* m, float* v,
-                     uint16_t* p, const UpdateConsts& k, const double* coef, cudaStream_t st) {
+                     uint16_t* p, const UpdateConsts& k, const double* coef, cudaStream_t st,
+                     bool early) {
   const int64_t groups = (n + kVec - 1) / kVec;
   const unsigned blocks = (unsigned)((groups + kUpdateThreads - 1) / kUpdateThreads);
-  reduce_adamw_kernel<R_T><<<blocks, kUpdateThreads, 0, st>>>(gp, n, w, m, v, p, k, coef);
+  LaunchCfg lc(blocks, kUpdateThreads, st, early);
+  (void)cudaLaunchKernelEx(&lc.cfg, reduce_adamw_kernel<R_T>, gp, n, w, m, v, p, k, coef);
 }
 
 int launch_update(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, float* w, float* m,
                   float* v, uint16_t* p, const UpdateConsts& k, const double* coef,
-                  cudaStream_t st) {
+                  cudaStream_t st, bool early) {
   if (n == 0) return SLIDEDP_OK;
   FAULT_POINT();
   // one instantiation per rank count: the R loads are fully unrolled (a runtime-R loop over a
   // 16-entry register array ran at 4.0 TB/s for R = 3 against 6.4+ TB/s unrolled)
   switch (R) {
-#define SLIDEDP_CASE(r) case r: launch_update_t<r>(gp, R, n, w, m, v, p, k, coef, st); break;
+#define SLIDEDP_CASE(r) case r: launch_update_t<r>(gp, R, n, w, m, v, p, k, coef, st, early); break;
     SLIDEDP_CASE(1) SLIDEDP_CASE(2) SLIDEDP_CASE(3) SLIDEDP_CASE(4) SLIDEDP_CASE(5) SLIDEDP_CASE(6)
     SLIDEDP_CASE(7) SLIDEDP_CASE(8) SLIDEDP_CASE(9) SLIDEDP_CASE(10) SLIDEDP_CASE(11)
     SLIDEDP_CASE(12) SLIDEDP_CASE(13) SLIDEDP_CASE(14) SLIDEDP_CASE(15) SLIDEDP_CASE(16)
@@ -124,10 +144,17 @@ int norm_chunk(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n, double in
   return SLIDEDP_OK;
 }
 
+// The finish kernel is queued so that it can be scheduled while the tile kernel before it is
+// still finishing (it waits for that kernel itself): hides its launch, 2-3 us per norm pass.
+static void launch_finish(const double* partials, int64_t count, double max_norm, double* scalars,
+                          cudaStream_t st) {
+  LaunchCfg lc(1, kFinishThreads, st, /*early=*/true);
+  (void)cudaLaunchKernelEx(&lc.cfg, grad_norm_finish_kernel, partials, count, max_norm, scalars);
+}
+
 int norm_finish(slidedp_ctx* ctx, double max_norm, cudaStream_t st) {
   FAULT_POINT();
-  grad_norm_finish_kernel<<<1, kFinishThreads, 0, st>>>(ctx->partials, ctx->partials_used,
-                                                        max_norm, ctx->scalars);
+  launch_finish(ctx->partials, ctx->partials_used, max_norm, ctx->scalars, st);
   ctx->launches += 1;
   CU_AFTER_LAUNCH();
   ctx->norm_issued = true;
@@ -205,7 +232,7 @@ int slidedp_grad_norm_finish_from(slidedp_ctx* ctx, const double* tile_sums, int
   if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   FAULT_POINT();
-  grad_norm_finish_kernel<<<1, kFinishThreads, 0, st>>>(tile_sums, count, max_norm, ctx->scalars);
+  launch_finish(tile_sums, count, max_norm, ctx->scalars, st);
   ctx->launches += 1;
   CU_AFTER_LAUNCH();
   ctx->norm_issued = true;
@@ -236,7 +263,7 @@ int slidedp_reduce_adamw_chunk(slidedp_ctx* ctx, const void* const* grads_bf16, 
   if (!guard.ok) return cuda_fail(ctx, cudaErrorInvalidDevice);
   return launch_update(ctx, gp, R, n, master, m, v, static_cast<uint16_t*>(param_bf16_out),
                        make_consts(hp), clip ? ctx->scalars + 2 : nullptr,
-                       static_cast<cudaStream_t>(cuda_stream));
+                       static_cast<cudaStream_t>(cuda_stream), /*early=*/true);
 }
 
 int slidedp_scatter_tile_sums(slidedp_ctx* ctx, const double* tile_sums, int64_t count,

@@ -214,6 +214,7 @@ template <int R, int UNROLL = (R >= 6) ? 1 : (R >= 3 ? 2 : 4)>
 __global__ void __launch_bounds__(kNormThreads)
 grad_sumsq_tiles_kernel(GradPtrs gp, int64_t n, float inv_R, double* __restrict__ partials) {
   __shared__ double warp_sum[kNormThreads / 32];
+  wait_for_previous_kernel();      // the gradients (and the tile-sum slots) may come from it
   const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
   for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
     const int64_t tbase = tile * kNormTile + (int64_t)threadIdx.x * kNormVec;
@@ -300,6 +301,7 @@ __global__ void __launch_bounds__(kNormThreads)
 grad_sumsq_tiles_r1_kernel(const uint16_t* __restrict__ g, int64_t n, float inv_R,
                            double* __restrict__ partials) {
   __shared__ double warp_sum[kDeepTiles][kNormThreads / 32];
+  wait_for_previous_kernel();
   const int64_t ntiles = (n + kNormTile - 1) / kNormTile;
   const int64_t first = (int64_t)blockIdx.x * kDeepTiles;
   uint4 raw[kDeepTiles][kNormIters];

@@ -84,18 +84,21 @@ static int launch_update_bcast(slidedp_ctx* ctx, const GradPtrs& gp, int R, int6
   return SLIDEDP_OK;
 }
 
-// One instantiation per rank count (R is validated to 1..16 before this is reached).
+// One instantiation per rank count (R is validated to 1..16 before this is reached). Queued so
+// that the kernel can be scheduled while the previous kernel of the stream is finishing (it waits
+// for that kernel itself before its first load).
 void launch_sumsq(const GradPtrs& gp, int R, int64_t n, float inv_R, double* tile_sums,
                   unsigned blocks, cudaStream_t st) {
   if (R == 1) {   // single rank: two tiles per block, every load of a tile in flight (same bits)
-    grad_sumsq_tiles_r1_kernel<<<(blocks + kDeepTiles - 1) / kDeepTiles, kNormThreads, 0, st>>>(
-        gp.p[0], n, inv_R, tile_sums);
+    LaunchCfg lc((blocks + kDeepTiles - 1) / kDeepTiles, kNormThreads, st, /*early=*/true);
+    (void)cudaLaunchKernelEx(&lc.cfg, grad_sumsq_tiles_r1_kernel, gp.p[0], n, inv_R, tile_sums);
     return;
   }
+  LaunchCfg lc(blocks, kNormThreads, st, /*early=*/true);
   switch (R) {
 #define SLIDEDP_CASE(r) \
-  case r: grad_sumsq_tiles_kernel<r><<<blocks, kNormThreads, 0, st>>>(gp, n, inv_R, tile_sums); break;
-    SLIDEDP_CASE(1) SLIDEDP_CASE(2) SLIDEDP_CASE(3) SLIDEDP_CASE(4) SLIDEDP_CASE(5) SLIDEDP_CASE(6)
+  case r: (void)cudaLaunchKernelEx(&lc.cfg, grad_sumsq_tiles_kernel<r>, gp, n, inv_R, tile_sums); break;
+    SLIDEDP_CASE(2) SLIDEDP_CASE(3) SLIDEDP_CASE(4) SLIDEDP_CASE(5) SLIDEDP_CASE(6)
     SLIDEDP_CASE(7) SLIDEDP_CASE(8) SLIDEDP_CASE(9) SLIDEDP_CASE(10) SLIDEDP_CASE(11)
     SLIDEDP_CASE(12) SLIDEDP_CASE(13) SLIDEDP_CASE(14) SLIDEDP_CASE(15) SLIDEDP_CASE(16)
 #undef SLIDEDP_CASE

@@ -349,6 +349,7 @@ int slidedp_stream_layers(slidedp_ctx* ctx, const slidedp_layer* layers, int num
     CU(cudaEventRecord(ctx->ev_norm_done, ctx->s_compute));
     for (int l = 0; l < num_layers; ++l) {
       const slidedp_layer& L = layers[l];
+      if (L.n == 0) continue;                  // nothing to stream (and no slot re-layout for it)
       int64_t nchunks = 0;
       const int marks = stats ? ((l == first ? kMarkFirst : 0) | (l == last ? kMarkLast : 0)) : 0;
       int r2 = enqueue_stream_step(ctx, L.grads_bf16, R, L.n, L.host_master, L.host_m, L.host_v,

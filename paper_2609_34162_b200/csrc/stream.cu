@@ -80,7 +80,7 @@ int enqueue_chunks(slidedp_ctx* ctx, const GradPtrs& gp, int R, int64_t n_total,
 int enqueue_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, int64_t n_total,
                         float* host_master, float* host_m, float* host_v, void* param_bf16_out,
                         int64_t chunk_elems, int nbuf, int norm_ready, const slidedp_hparams* hp,
-                        bool synchronous, int marks, int64_t* nchunks_out) {
+                        bool synchronous, int marks, int64_t* nchunks_out, int64_t cap_hint = 0) {
   if (!ctx || n_total < 0) return SLIDEDP_ERR_INVALID_ARG;
   int rc = check_hparams(hp);
   if (rc != SLIDEDP_OK) return rc;
@@ -109,7 +109,10 @@ int enqueue_stream_step(slidedp_ctx* ctx, const void* const* grads_bf16, int R, 
   }
 
   // slots: nbuf x {master, m, v} x cap floats
-  const int64_t cap = chunk_elems < n_total ? chunk_elems : ((n_total + 7) / 8) * 8;
+  // (a multi-layer call passes the slot capacity of its largest layer, so that small layers do
+  // not force a new layout and a drain in the middle of the step)
+  const int64_t own_cap = chunk_elems < n_total ? chunk_elems : ((n_total + 7) / 8) * 8;
+  const int64_t cap = cap_hint > own_cap ? cap_hint : own_cap;
   const size_t need = (size_t)nbuf * 3 * (size_t)cap * sizeof(float);
   if (ctx->budget && need > ctx->budget) return SLIDEDP_ERR_BUDGET;
   const bool relayout = cap != ctx->ring_cap || nbuf != ctx->ring_nbuf || need > ctx->slot_bytes;
@@ -320,13 +323,11 @@ int slidedp_stream_layers(slidedp_ctx* ctx, const slidedp_layer* layers, int num
       if (!pinned) return SLIDEDP_ERR_NOT_PINNED;
     }
   }
-  {
-    int64_t biggest = 0;
-    for (int l = 0; l < num_layers; ++l) if (layers[l].n > biggest) biggest = layers[l].n;
-    const int64_t cap = chunk_elems < biggest ? chunk_elems : ((biggest + 7) / 8) * 8;
-    if (ctx->budget && (size_t)nbuf * 3 * (size_t)cap * sizeof(float) > ctx->budget)
-      return SLIDEDP_ERR_BUDGET;
-  }
+  int64_t biggest = 0;
+  for (int l = 0; l < num_layers; ++l) if (layers[l].n > biggest) biggest = layers[l].n;
+  const int64_t cap_all = chunk_elems < biggest ? chunk_elems : ((biggest + 7) / 8) * 8;
+  if (ctx->budget && (size_t)nbuf * 3 * (size_t)cap_all * sizeof(float) > ctx->budget)
+    return SLIDEDP_ERR_BUDGET;
 
   int64_t chunks = 0;
   ctx->ring_busy = true;
@@ -354,7 +355,7 @@ int slidedp_stream_layers(slidedp_ctx* ctx, const slidedp_layer* layers, int num
       const int marks = stats ? ((l == first ? kMarkFirst : 0) | (l == last ? kMarkLast : 0)) : 0;
       int r2 = enqueue_stream_step(ctx, L.grads_bf16, R, L.n, L.host_master, L.host_m, L.host_v,
                                    L.param_bf16_out, chunk_elems, nbuf, /*norm_ready=*/1, hp,
-                                   /*synchronous=*/false, marks, &nchunks);
+                                   /*synchronous=*/false, marks, &nchunks, cap_all);
       if (r2 != SLIDEDP_OK) return r2;
       chunks += nchunks;
     }

@@ -351,6 +351,11 @@ def run_cuda(args):
             route = cpu_route_report(ctx, sd, W, torch, dev)
         except Exception as exc:
             route = {"error": repr(exc)}
+        # both delivery routes side by side where the host-resident configuration is reported
+        if isinstance(host, dict) and isinstance(route, dict) and "delivery" in host and "delivery" in route:
+            host["delivery"]["routes"] = {
+                "fp32_h2d_gpu_cast (slidedp_deliver_params)": route["delivery"]["fp32_h2d_gpu_cast"],
+                "cpu_cast_bf16_h2d (the paper's route, baseline/cpu_route)": route["delivery"]["cpu_cast_bf16_h2d"]}
         cpu = cpu_baseline(W, torch, np, wl, grads, layer)
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -246,6 +246,23 @@ def test_every_device_resident_entry_point_survives_a_failed_runtime_call(ctx, s
         got["nc2"] = ctx.slidedp_grad_norm_finish_from(tiles, tiles.numel(), case.kw["max_norm"], fetch=True)
     assert _sweep(ctx, sd, finish_from, nothing) == 3
     assert got["nc2"] == got["nc"]
+    # the sharded step's entry points and the roofline probe
+    dsts = [torch.zeros_like(tiles), torch.zeros_like(tiles)]
+    assert _sweep(ctx, sd, lambda: ctx.slidedp_scatter_tile_sums(tiles, tiles.numel(), dsts), nothing) == 1
+    torch.cuda.synchronize()
+    assert all(torch.equal(d, tiles) for d in dsts)
+    b = [torch.from_numpy(x).cuda() for x in (case.w0, case.m0, case.v0)]
+    outs = [torch.zeros(n, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    torch.cuda.synchronize()
+    assert _sweep(ctx, sd, lambda: ctx.slidedp_reduce_adamw_chunk_bcast(case.dg, n, *b, outs, hp),
+                  nothing) == 1
+    torch.cuda.synchronize()
+    case.check_state(*(parity.f32(x) for x in b), parity.u16(outs[1]))
+    assert _sweep(ctx, sd, lambda: ctx.slidedp_ipc_export(outs[0]), nothing) == 2
+    assert len(ctx.slidedp_ipc_export(outs[0])) == sd.IPC_HANDLE_BYTES
+    assert _sweep(ctx, sd, lambda: ctx.slidedp_hbm_mix_probe(case.dg, n, *b, outs[0], 1), nothing) >= 1
+    torch.cuda.synchronize()
+    case.check_state(*(parity.f32(x) for x in b), parity.u16(outs[1]))      # the probe left the state alone
 
 
 def test_non_finite_hyper_parameters_are_rejected(ctx, sd):
